@@ -1,0 +1,211 @@
+#include "forward.hpp"
+
+#include <algorithm>
+#include <cstring>
+
+#include "kernels.cuh"
+
+namespace relaygr {
+
+namespace {
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+std::string cuda_msg(const char *what, cudaError_t e) { return std::string(what) + ": " + cudaGetErrorString(e); }
+}  // namespace
+
+Forward::~Forward()
+{
+    for (int i = 0; i < kSlots; ++i) if (slot_event[i]) cudaEventDestroy(slot_event[i]);
+    if (staging) cudaFreeHost(staging);
+}
+
+int Forward::init_device(int dev, std::string &err)
+{
+    device = dev;
+    cudaDeviceProp prop;
+    cudaError_t e = cudaGetDeviceProperties(&prop, dev);
+    if (e != cudaSuccess) { err = cuda_msg("cudaGetDeviceProperties", e); return RELAYGR_E_CUDA; }
+    if (prop.major != 10) { err = "this library is built for sm_100a (B200) only"; return RELAYGR_E_UNSUPPORTED; }
+    n_sms = prop.multiProcessorCount;
+    e = cudaMallocHost((void **)&staging, kSlots * kSlotBytes);
+    if (e != cudaSuccess) { staging = nullptr; err = cuda_msg("cudaMallocHost (metadata staging)", e); return RELAYGR_E_CUDA; }
+    for (int i = 0; i < kSlots; ++i) {
+        e = cudaEventCreateWithFlags(&slot_event[i], cudaEventDisableTiming);
+        if (e != cudaSuccess) { err = cuda_msg("cudaEventCreate", e); return RELAYGR_E_CUDA; }
+    }
+    return RELAYGR_OK;
+}
+
+WorkspaceLayout Forward::layout(int64_t rows, int64_t users, int64_t pages) const
+{
+    WorkspaceLayout l{};
+    const size_t d = (size_t)cfg.d_model, F = (size_t)cfg.d_ff, es = esize();
+    const size_t r = (size_t)rows + 128;    // slack so that 128-row tiles may read past the last row
+    size_t at = 0;
+    auto take = [&](size_t bytes) { const size_t o = at; at = align_up(at + bytes, 1024); return o; };
+    l.x = take(r * d * 4);
+    l.a = take(r * d * es);
+    l.q = take(r * d * es);
+    l.k = take(r * d * es);
+    l.v = take(r * d * es);
+    l.att = take(r * d * es);
+    l.hid = take(r * F * es);
+    l.partial_bytes = (size_t)kMaxSplitTiles * 128 * (size_t)(cfg.d_head + 2) * 4;
+    l.partial = take(l.partial_bytes);
+    const size_t n_items = (size_t)cfg.n_heads * ((size_t)rows / 128 + (size_t)users + 1) + 2 * (size_t)kMaxSplitTiles;
+    l.meta_bytes = 4 * (((size_t)users + 1) * 5 + (size_t)users * (sizeof(SeqDesc) / 4) + (size_t)pages + n_items * (sizeof(AttnWork) / 4) + 64);
+    l.meta = take(l.meta_bytes);
+    l.total = at;
+    return l;
+}
+
+int Forward::check_capacity(const CallDesc &call, std::string &err) const
+{
+    if (!ws) { err = "no workspace set (relaygr_set_workspace)"; return RELAYGR_E_NOSPACE; }
+    const WorkspaceLayout l = layout(call.n_rows, (int64_t)call.seqs.size(), (int64_t)call.page_table.size());
+    if (l.total > ws_bytes) { err = "workspace too small for this call (see relaygr_workspace_bytes)"; return RELAYGR_E_NOSPACE; }
+    return RELAYGR_OK;
+}
+
+int Forward::upload(const std::vector<int32_t> &blob, size_t dst_off, cudaStream_t stream, std::string &err)
+{
+    const size_t bytes = blob.size() * 4;
+    cudaError_t e;
+    if (bytes <= kSlotBytes) {
+        const int s = next_slot;
+        next_slot = (next_slot + 1) % kSlots;
+        if (slot_used[s]) {
+            e = cudaEventSynchronize(slot_event[s]);       // only waits if kSlots calls are still in flight
+            if (e != cudaSuccess) { err = cuda_msg("cudaEventSynchronize", e); return RELAYGR_E_CUDA; }
+        }
+        char *src = staging + (size_t)s * kSlotBytes;
+        std::memcpy(src, blob.data(), bytes);
+        e = cudaMemcpyAsync(ws + dst_off, src, bytes, cudaMemcpyHostToDevice, stream);
+        if (e == cudaSuccess) e = cudaEventRecord(slot_event[s], stream);
+        slot_used[s] = true;
+    } else {
+        e = cudaMemcpyAsync(ws + dst_off, blob.data(), bytes, cudaMemcpyHostToDevice, stream);   // pageable: staged by the runtime
+    }
+    if (e != cudaSuccess) { err = cuda_msg("metadata upload", e); return RELAYGR_E_CUDA; }
+    return RELAYGR_OK;
+}
+
+int Forward::gather(const int32_t *ids, int64_t n, void *out, cudaStream_t stream, std::string &err)
+{
+    cudaError_t e;
+    if (cfg.dtype == RELAYGR_DTYPE_F32)
+        e = launch_gather_rows<float>((const float *)w.emb, cfg.vocab, cfg.d_model, ids, n, (float *)out, stream, &launches);
+    else
+        e = launch_gather_rows<__nv_bfloat16>((const __nv_bfloat16 *)w.emb, cfg.vocab, cfg.d_model, ids, n, (__nv_bfloat16 *)out,
+                                              stream, &launches);
+    if (e != cudaSuccess) { err = cuda_msg("gather", e); return RELAYGR_E_CUDA; }
+    return RELAYGR_OK;
+}
+
+int Forward::run(const CallDesc &call, float *scores, cudaStream_t stream, std::string &err)
+{
+    if (cfg.dtype == RELAYGR_DTYPE_F32) return run_t<float>(call, scores, stream, err);
+    return run_t<__nv_bfloat16>(call, scores, stream, err);
+}
+
+template <typename T>
+int Forward::run_t(const CallDesc &call, float *scores, cudaStream_t stream, std::string &err)
+{
+    const int B = (int)call.seqs.size();
+    const int64_t R = call.n_rows;
+    if (R == 0) return RELAYGR_OK;
+    const int d = cfg.d_model, F = cfg.d_ff, L = cfg.n_layers, H = cfg.n_heads;
+    const WorkspaceLayout lay = layout(R, B, (int64_t)call.page_table.size());
+
+    // ---- metadata blob: row_off | seg_off x3 | score_off | SeqDesc[] | page table
+    std::vector<int32_t> blob;
+    auto put = [&](const int32_t *p, size_t n) { const size_t o = blob.size(); blob.insert(blob.end(), p, p + n); return o; };
+    std::vector<int32_t> row_off((size_t)B + 1);
+    for (int i = 0; i < B; ++i) row_off[(size_t)i] = call.seqs[(size_t)i].q_row0;
+    row_off[(size_t)B] = (int32_t)R;
+    const size_t o_row = put(row_off.data(), (size_t)B + 1);
+    size_t o_seg[3] = {0, 0, 0};
+    for (int s = 0; s < 3; ++s) if (call.seg_off[s]) o_seg[s] = put(call.seg_off[s], (size_t)B + 1);
+    const size_t o_score = call.score_off ? put(call.score_off, (size_t)B + 1) : 0;
+    const size_t o_seq = put(reinterpret_cast<const int32_t *>(call.seqs.data()), (size_t)B * (sizeof(SeqDesc) / 4));
+    const size_t o_pt = call.page_table.empty() ? 0 : put(call.page_table.data(), call.page_table.size());
+    if (blob.size() * 4 > lay.meta_bytes) { err = "internal: metadata larger than its workspace region"; return RELAYGR_E_NOSPACE; }
+    int rc = upload(blob, lay.meta, stream, err);
+    if (rc) return rc;
+
+    const int32_t *meta = reinterpret_cast<const int32_t *>(ws + lay.meta);
+    const int32_t *d_row_off = meta + o_row;
+    const SeqDesc *d_seqs = reinterpret_cast<const SeqDesc *>(meta + o_seq);
+    RowSource src{};
+    for (int s = 0; s < 3; ++s) {
+        const bool on = call.seg_off[s] && call.seg_off[s][B] > 0;
+        src.ids[s] = on ? call.seg_ids[s] : nullptr;
+        src.off[s] = on ? meta + o_seg[s] : nullptr;
+    }
+    src.row_off = d_row_off;
+    src.n_users = B;
+
+    float *x = reinterpret_cast<float *>(ws + lay.x);
+    T *a = reinterpret_cast<T *>(ws + lay.a), *q = reinterpret_cast<T *>(ws + lay.q);
+    T *kl = reinterpret_cast<T *>(ws + lay.k), *vl = reinterpret_cast<T *>(ws + lay.v);
+    T *att = reinterpret_cast<T *>(ws + lay.att), *hid = reinterpret_cast<T *>(ws + lay.hid);
+    const bool preinfer = call.mode == MODE_PREINFER;
+
+    cudaError_t e = cudaSuccess;
+    auto ck = [&](const char *what) -> bool { if (e != cudaSuccess) { err = cuda_msg(what, e); return false; } return true; };
+
+    for (int l = 0; l < L; ++l) {
+        const float *g1 = w.ln1_g + (size_t)l * d, *b1n = w.ln1_b + (size_t)l * d;
+        if (l == 0) e = launch_gather_ln<T>((const T *)w.emb, cfg.vocab, d, src, R, g1, b1n, cfg.ln_eps, x, a, stream, &launches);
+        else e = launch_layernorm<T>(x, d, R, g1, b1n, cfg.ln_eps, a, stream, &launches);
+        if (!ck("LayerNorm 1")) return RELAYGR_E_CUDA;
+
+        // fused QKV projection; the last pre-infer layer only needs K and V (psi is K/V alone)
+        const bool kv_only = preinfer && l == L - 1;
+        Epilogue ep{};
+        ep.mode = EPI_QKV;
+        ep.col0 = kv_only ? d : 0;
+        ep.bias = w.b_qkv ? w.b_qkv + (size_t)l * 3 * d + ep.col0 : nullptr;
+        ep.d_model = d;
+        ep.q = q; ep.k_lin = kl; ep.v_lin = vl;
+        ep.seqs = d_seqs; ep.row_off = d_row_off; ep.n_users = B;
+        PagedKV paged{};
+        if (call.pool_slab) {
+            paged.slab = call.pool_slab; paged.pt = meta + o_pt; paged.n_layers = L; paged.d_model = d; paged.layer = l;
+        }
+        if (preinfer) ep.paged = paged;
+        const T *Wqkv = (const T *)w.w_qkv + ((size_t)l * 3 * d + ep.col0) * d;
+        e = launch_gemm_simt<T>(a, Wqkv, R, 3 * d - ep.col0, d, ep, stream, &launches);
+        if (!ck("QKV projection")) return RELAYGR_E_CUDA;
+        if (kv_only) break;
+
+        e = launch_attention_simt<T>(q, kl, vl, paged, d_seqs, d_row_off, B, R, H, cfg.d_head, att, stream, &launches);
+        if (!ck("attention")) return RELAYGR_E_CUDA;
+
+        Epilogue eo{};
+        eo.mode = EPI_RESID; eo.bias = w.b_o ? w.b_o + (size_t)l * d : nullptr; eo.resid = x; eo.out_f32 = x;
+        e = launch_gemm_simt<T>(att, (const T *)w.w_o + (size_t)l * d * d, R, d, d, eo, stream, &launches);
+        if (!ck("output projection")) return RELAYGR_E_CUDA;
+
+        e = launch_layernorm<T>(x, d, R, w.ln2_g + (size_t)l * d, w.ln2_b + (size_t)l * d, cfg.ln_eps, a, stream, &launches);
+        if (!ck("LayerNorm 2")) return RELAYGR_E_CUDA;
+
+        Epilogue e1{};
+        e1.mode = EPI_STORE; e1.silu = 1; e1.bias = w.b1 ? w.b1 + (size_t)l * F : nullptr; e1.out = hid;
+        e = launch_gemm_simt<T>(a, (const T *)w.w1 + (size_t)l * F * d, R, F, d, e1, stream, &launches);
+        if (!ck("FFN 1")) return RELAYGR_E_CUDA;
+
+        Epilogue e2{};
+        e2.mode = EPI_RESID; e2.bias = w.b2 ? w.b2 + (size_t)l * d : nullptr; e2.resid = x; e2.out_f32 = x;
+        e = launch_gemm_simt<T>(hid, (const T *)w.w2 + (size_t)l * d * F, R, d, F, e2, stream, &launches);
+        if (!ck("FFN 2")) return RELAYGR_E_CUDA;
+    }
+
+    if (!preinfer && call.score_off && call.score_off[B] > 0) {
+        e = launch_score(x, d, d_seqs, B, call.score_off[B], meta + o_score, w.lnf_g, w.lnf_b, cfg.ln_eps, w.w_score, w.b_score,
+                         scores, stream, &launches);
+        if (!ck("scoring head")) return RELAYGR_E_CUDA;
+    }
+    return RELAYGR_OK;
+}
+
+}  // namespace relaygr

@@ -1,0 +1,76 @@
+// Orchestration of one forward pass (pre-infer, rank on cache, or full inference):
+// builds the per-call metadata, uploads it, and enqueues the kernels layer by layer.
+#pragma once
+
+#include <cstdint>
+#include <string>
+#include <vector>
+
+#include <cuda_runtime.h>
+
+#include "../../include/relaygr.h"
+#include "internal.cuh"
+
+namespace relaygr {
+
+enum CallMode { MODE_PREINFER = 0, MODE_RANK = 1, MODE_FULL = 2 };
+
+struct CallDesc {
+    int mode = MODE_RANK;
+    std::vector<SeqDesc> seqs;
+    std::vector<int32_t> page_table;
+    int64_t n_rows = 0;
+    const int32_t *seg_ids[3] = {nullptr, nullptr, nullptr};   // device
+    const int32_t *seg_off[3] = {nullptr, nullptr, nullptr};   // host, [n_users + 1]
+    const int32_t *score_off = nullptr;                        // host, [n_users + 1]
+    void *pool_slab = nullptr;
+    int64_t pool_pages = 0;
+};
+
+struct WorkspaceLayout {
+    size_t x, a, q, k, v, att, hid, partial, meta, total;
+    size_t meta_bytes, partial_bytes;
+};
+
+// One unit of tensor-core attention work: a 128-row query tile of one head of one
+// user against a contiguous range of that user's 128-key blocks.
+struct AttnWork {
+    int32_t seq, head, q0, n_q;          // query rows q0 .. q0+n_q-1 of the user (local index)
+    int32_t blk0, blk1;                  // key blocks [blk0, blk1) in the order: paged blocks, then linear blocks
+    int32_t partial_slot;                // >= 0: write (m, l, O) partials here instead of the output
+    int32_t n_splits;
+};
+
+struct Forward {
+    relaygr_model_cfg cfg{};
+    relaygr_weights w{};
+    char *ws = nullptr;
+    size_t ws_bytes = 0;
+    int64_t launches = 0;
+    int device = 0;
+    int n_sms = 148;
+
+    // pinned staging ring for the per-call metadata
+    static constexpr int kSlots = 4;
+    static constexpr size_t kSlotBytes = 2u << 20;
+    char *staging = nullptr;
+    cudaEvent_t slot_event[kSlots] = {};
+    bool slot_used[kSlots] = {};
+    int next_slot = 0;
+
+    ~Forward();
+    int init_device(int dev, std::string &err);
+    WorkspaceLayout layout(int64_t rows, int64_t users, int64_t pages) const;
+    int check_capacity(const CallDesc &call, std::string &err) const;
+    int run(const CallDesc &call, float *scores, cudaStream_t stream, std::string &err);
+    int gather(const int32_t *ids, int64_t n, void *out, cudaStream_t stream, std::string &err);
+
+    size_t esize() const { return cfg.dtype == RELAYGR_DTYPE_F32 ? 4 : 2; }
+    static constexpr int64_t kMaxSplitTiles = 1536;   // capacity of the split-KV partial buffer, in 128-row tiles
+
+private:
+    template <typename T> int run_t(const CallDesc &call, float *scores, cudaStream_t stream, std::string &err);
+    int upload(const std::vector<int32_t> &blob, size_t dst_off, cudaStream_t stream, std::string &err);
+};
+
+}  // namespace relaygr

@@ -1,0 +1,87 @@
+// Structures shared by the host runtime and the kernels.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace relaygr {
+
+// One user of a call.  Rows are the token rows the call computes (activations are
+// dense [n_rows, d], users back to back).  Keys come from two places: "paged" keys
+// (the pool, through the page table) at sequence positions 0 .. n_paged-1, and
+// "linear" keys (rows of the call's transient K/V buffers) at positions
+// lin_pos0 .. lin_pos0+n_lin-1.  Mask: a query at position t < causal_end sees
+// keys at positions <= t; a query at t >= causal_end (a candidate) sees keys at
+// positions < causal_end plus its own K/V row.
+struct SeqDesc {
+    int32_t q_row0, n_q, q_pos0;
+    int32_t n_paged, pt_base;
+    int32_t lin_row0, n_lin, lin_pos0;
+    int32_t causal_end;
+    int32_t score_row0, n_score, score_out0;
+};
+
+// Where the token ids of the rows come from: up to three jagged segments per user, in order.
+struct RowSource {
+    const int32_t *ids[3];   // device id arrays (nullptr = segment absent)
+    const int32_t *off[3];   // device offsets [n_users + 1] of each segment
+    const int32_t *row_off;  // device [n_users + 1]
+    int32_t n_users;
+};
+
+// Addressing of the paged pool: page = [L][K|V][64][d].
+struct PagedKV {
+    void *slab;
+    const int32_t *pt;       // device page table (all users of the call, concatenated)
+    int32_t n_layers, d_model, layer;
+};
+
+enum EpiMode : int32_t { EPI_STORE = 0, EPI_RESID = 1, EPI_QKV = 2 };
+
+// What a GEMM does with its fp32 accumulators: C[m, n] = sum_k A[m,k] W[n,k].
+struct Epilogue {
+    int32_t mode;
+    int32_t silu;                 // EPI_STORE: apply SiLU after the bias
+    const float *bias;            // [N] (already offset to this layer), may be nullptr
+    void *out;                    // EPI_STORE: [M, N] in the model dtype
+    const float *resid;           // EPI_RESID: fp32 [M, N] read ...
+    float *out_f32;               // ... and fp32 [M, N] written (may alias resid)
+    // EPI_QKV: column c of the full [3d] output goes to q (c < d), K (d <= c < 2d) or V.
+    int32_t col0;                 // first output column this GEMM computes (0, or d for K/V only)
+    int32_t d_model;
+    void *q;                      // [M, d]
+    void *k_lin, *v_lin;          // [M, d] transient K/V (used when paged.slab == nullptr)
+    PagedKV paged;                // else K/V rows are scattered into pages
+    const SeqDesc *seqs;          // per-user descriptors (paged scatter needs row -> user -> page)
+    const int32_t *row_off;
+    int32_t n_users;
+};
+
+__device__ __forceinline__ int find_user(const int32_t *row_off, int n_users, int row)
+{
+    // largest u with row_off[u] <= row
+    int lo = 0, hi = n_users;
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (row_off[mid] <= row) lo = mid; else hi = mid;
+    }
+    return lo;
+}
+
+__device__ __forceinline__ size_t page_elem_offset(const PagedKV &p, int page, int kv, int slot)
+{
+    return ((((size_t)page * p.n_layers + p.layer) * 2 + kv) * 64 + slot) * (size_t)p.d_model;
+}
+
+template <typename T> struct Num;
+template <> struct Num<float> {
+    static __device__ __forceinline__ float to_f(float v) { return v; }
+    static __device__ __forceinline__ float from_f(float v) { return v; }
+};
+template <> struct Num<__nv_bfloat16> {
+    static __device__ __forceinline__ float to_f(__nv_bfloat16 v) { return __bfloat162float(v); }
+    static __device__ __forceinline__ __nv_bfloat16 from_f(float v) { return __float2bfloat16_rn(v); }
+};
+
+}  // namespace relaygr

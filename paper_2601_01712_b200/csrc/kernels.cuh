@@ -1,0 +1,45 @@
+// Launchers of the device kernels.  Every launcher enqueues on `stream`, returns the
+// cudaError_t of the launch and adds the number of kernels it launched to *launches.
+#pragma once
+
+#include "internal.cuh"
+
+namespace relaygr {
+
+// ---- memory-bound steps (CUDA cores, vectorised loads, warp-shuffle reductions) ----------------
+
+// out[i, :] = emb[ids[i], :], a bit-exact row copy.
+template <typename T>
+cudaError_t launch_gather_rows(const T *emb, int64_t vocab, int d, const int32_t *ids, int64_t n, T *out,
+                               cudaStream_t stream, int64_t *launches);
+
+// x[r, :] = emb[id(r), :] widened to fp32 (the residual stream); a[r, :] = LN(x[r, :]; g, b) in T.
+template <typename T>
+cudaError_t launch_gather_ln(const T *emb, int64_t vocab, int d, RowSource src, int64_t n_rows,
+                             const float *g, const float *b, float eps, float *x, T *a,
+                             cudaStream_t stream, int64_t *launches);
+
+// a[r, :] = LN(x[r, :]; g, b) in T.
+template <typename T>
+cudaError_t launch_layernorm(const float *x, int d, int64_t n_rows, const float *g, const float *b, float eps, T *a,
+                             cudaStream_t stream, int64_t *launches);
+
+// scores[score_out0 + i] = LN(x[score_row0 + i]; g, b) . w + bias for every user's candidate rows.
+cudaError_t launch_score(const float *x, int d, const SeqDesc *seqs, int n_users, int64_t n_scores_total,
+                         const int32_t *score_off, const float *g, const float *b, float eps,
+                         const float *w, const float *bias, float *scores, cudaStream_t stream, int64_t *launches);
+
+// ---- CUDA-core GEMM and attention (the fp32 model) ---------------------------------------------
+
+// C[m, n] = sum_k A[m, k] W[n, k], m < M, n < N, then `epi`.
+template <typename T>
+cudaError_t launch_gemm_simt(const T *A, const T *W, int64_t M, int N, int K, const Epilogue &epi,
+                             cudaStream_t stream, int64_t *launches);
+
+// One warp per (row, head): softmax attention under the SeqDesc mask.  out [n_rows, d] in T.
+template <typename T>
+cudaError_t launch_attention_simt(const T *q, const T *k_lin, const T *v_lin, PagedKV paged, const SeqDesc *seqs,
+                                  const int32_t *row_off, int n_users, int64_t n_rows, int n_heads, int d_head,
+                                  T *out, cudaStream_t stream, int64_t *launches);
+
+}  // namespace relaygr

@@ -1,0 +1,234 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU checker on the
+same seeded inputs.  Integer / byte work (gather, page indexing, tier copies) must be
+bit-exact; scores within 1e-4 (fp32 model) or 2e-2 (bf16 model) max-abs."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2601_01712_b200 import synth
+from tests.helpers import TOL_BF16, TOL_F32, max_abs_err, oracle_model, oracle_scores, small_bf16_shape
+
+pytestmark = pytest.mark.gpu
+
+
+def _runtime():
+    from paper_2601_01712_b200 import binding, runtime
+    return binding, runtime
+
+
+def _setup(shape, seed, batch, hbm_pages=None, host_pages=0, page_ids=None):
+    B, rt = _runtime()
+    w = synth.make_weights(shape, seed)
+    model = rt.Model(shape, w)
+    n_pages = [synth.pages_for(batch.prefix_off[i + 1] - batch.prefix_off[i]) for i in range(batch.n_users)]
+    total = sum(n_pages)
+    pool = rt.KvPool(model, hbm_pages or total + 3, host_pages)
+    rows = int(batch.prefix_off[-1] + batch.short_off[-1] + batch.cand_off[-1])
+    model.reserve(rows, batch.n_users, total)
+    for i in range(batch.n_users):
+        pool.alloc(batch.users[i], batch.prefix_off[i + 1] - batch.prefix_off[i], None if page_ids is None else page_ids[i])
+    db = rt.DeviceBatch(batch, model.device)
+    return w, model, pool, db
+
+
+def _tiny_batch(shape, seed, p, s, c):
+    rng = np.random.default_rng(seed)
+    return synth.make_batch(synth.ZipfIds(shape.vocab, 1.1), rng, p, s, c)
+
+
+# ---------------------------------------------------------------- config 1: tiny fp32 model
+def test_config1_fp32_preinfer_rank_full():
+    wl = synth.workload(1)
+    shape = wl.model
+    rng = np.random.default_rng(wl.seed)
+    batch = synth.config1_batch(synth.ZipfIds(shape.vocab, wl.zipf_a), rng)
+    w, model, pool, db = _setup(shape, wl.seed, batch)
+    om = oracle_model(shape, w)
+
+    pool.preinfer(db)
+    scores = pool.rank(db)
+    full = model.rank_full(db)
+    torch.cuda.synchronize()
+
+    # psi: per-layer K / V rows of the prefix
+    for i in range(batch.n_users):
+        p, _, _ = batch.user_slices(i)
+        K, V = om.preinfer(p)
+        gK, gV = pool.read_kv(batch.users[i], len(p))
+        assert np.max(np.abs(gK.cpu().numpy().astype(np.float64) - K)) <= TOL_F32
+        assert np.max(np.abs(gV.cpu().numpy().astype(np.float64) - V)) <= TOL_F32
+    want = oracle_scores(om, batch)
+    assert max_abs_err(scores.cpu().numpy(), batch, want) <= TOL_F32
+    assert max_abs_err(full.cpu().numpy(), batch, want) <= TOL_F32
+    # the paper's relation: rank on cache ~= full inference
+    assert np.max(np.abs(scores.cpu().numpy() - full.cpu().numpy())) <= TOL_F32
+    assert model.launch_count() > 0
+    pool.close(); model.close()
+
+
+def test_gather_is_bit_exact_fp32_and_bf16():
+    _, rt = _runtime()
+    for shape in (synth.MODEL_TINY, small_bf16_shape()):
+        w = synth.make_weights(shape, 5)
+        model = rt.Model(shape, w)
+        rng = np.random.default_rng(9)
+        ids = synth.ZipfIds(shape.vocab, 1.1).draw(rng, 1000 + 37)
+        ids[:3] = [0, shape.vocab - 1, 1]
+        out = model.gather(torch.from_numpy(ids).to(model.device))
+        torch.cuda.synchronize()
+        if shape.dtype == synth.DTYPE_BF16:
+            got = out.view(torch.int16).cpu().numpy().view(np.uint16)
+            assert np.array_equal(got, w.bits["emb"][ids])
+        else:
+            assert np.array_equal(out.cpu().numpy().view(np.uint32), w.mat["emb"][ids].view(np.uint32))
+        model.close()
+
+
+# ---------------------------------------------------------------- jagged bf16 batches (several tiles, ragged tails)
+JAGGED = [
+    ([300, 129, 64, 1000], [5, 0, 70, 33], [130, 7, 0, 257]),
+    ([1, 63, 65, 128], [0, 1, 0, 130], [1, 0, 129, 3]),
+]
+
+
+@pytest.mark.parametrize("case", range(len(JAGGED)))
+def test_jagged_bf16_matches_checker(case):
+    p, s, c = JAGGED[case]
+    shape = small_bf16_shape()
+    batch = _tiny_batch(shape, 40 + case, p, s, c)
+    w, model, pool, db = _setup(shape, 21, batch)
+    om = oracle_model(shape, w)
+    pool.preinfer(db)
+    scores = pool.rank(db)
+    full = model.rank_full(db)
+    torch.cuda.synchronize()
+    for i in range(batch.n_users):
+        pp, _, _ = batch.user_slices(i)
+        K, V = om.preinfer(pp)
+        gK, gV = pool.read_kv(batch.users[i], len(pp))
+        assert np.max(np.abs(gK.float().cpu().numpy() - K)) <= 5e-2      # bf16 rows of magnitude ~1-4
+        assert np.max(np.abs(gV.float().cpu().numpy() - V)) <= 5e-2
+    want = oracle_scores(om, batch)
+    assert max_abs_err(scores.cpu().numpy(), batch, want) <= TOL_BF16
+    assert max_abs_err(full.cpu().numpy(), batch, want) <= TOL_BF16
+    pool.close(); model.close()
+
+
+def test_shuffled_page_table_changes_nothing():
+    """Pages scattered by a shuffled page table hold bit-identical rows and give bit-identical scores."""
+    shape = small_bf16_shape()
+    p, s, c = [700, 130, 2049], [17, 64, 3], [140, 200, 31]
+    batch = _tiny_batch(shape, 77, p, s, c)
+    counts = [synth.pages_for(x) for x in p]
+    res = []
+    for shuffled in (False, True):
+        ids = synth.shuffled_pages(np.random.default_rng(5), sum(counts) + 40, counts) if shuffled else None
+        w, model, pool, db = _setup(shape, 22, batch, hbm_pages=sum(counts) + 40, page_ids=ids)
+        pool.preinfer(db)
+        scores = pool.rank(db)
+        torch.cuda.synchronize()
+        if shuffled:
+            for i in range(batch.n_users):
+                assert np.array_equal(pool.pages(batch.users[i]), ids[i])
+        kv = [tuple(t.view(torch.int16).cpu().numpy() for t in pool.read_kv(batch.users[i], p[i])) for i in range(3)]
+        res.append((scores.cpu().numpy().copy(), kv))
+        pool.close(); model.close()
+    assert np.array_equal(res[0][0].view(np.uint32), res[1][0].view(np.uint32))
+    for a, b in zip(res[0][1], res[1][1]):
+        assert np.array_equal(a[0], b[0]) and np.array_equal(a[1], b[1])
+
+
+def test_preinfer_is_deterministic_and_rank_leaves_pages_untouched():
+    shape = small_bf16_shape()
+    batch = _tiny_batch(shape, 78, [500, 200], [10, 20], [100, 50])
+    w, model, pool, db = _setup(shape, 23, batch)
+    pool.preinfer(db)
+    torch.cuda.synchronize()
+    before = pool.slab.clone()
+    pool.rank(db)
+    torch.cuda.synchronize()
+    assert torch.equal(before, pool.slab)
+    # a second pre-infer of the same prefixes into fresh pages gives the same rows
+    for u in reversed(batch.users):      # so that the free list hands the same pages out again
+        pool.evict(u, False)
+    for i, u in enumerate(batch.users):
+        pool.alloc(u, batch.prefix_off[i + 1] - batch.prefix_off[i])
+    pool.preinfer(db)
+    torch.cuda.synchronize()
+    assert torch.equal(before, pool.slab)
+    pool.close(); model.close()
+
+
+def test_batch_equals_single_user_calls_and_candidate_independence():
+    B, rt = _runtime()
+    shape = small_bf16_shape()
+    batch = _tiny_batch(shape, 79, [400, 150], [12, 40], [200, 90])
+    w, model, pool, db = _setup(shape, 24, batch)
+    pool.preinfer(db)
+    scores = pool.rank(db).cpu().numpy().copy()
+    # user 1 alone, with only a slice of its candidates
+    one = synth.Batch(batch.users[1:2], batch.prefix_ids[400:], np.array([0, 150], np.int32),
+                      batch.short_ids[12:], np.array([0, 40], np.int32),
+                      batch.cand_ids[200 + 10:200 + 30], np.array([0, 20], np.int32))
+    s1 = pool.rank(rt.DeviceBatch(one, model.device)).cpu().numpy()
+    assert np.max(np.abs(s1 - scores[200 + 10:200 + 30])) <= 1e-5
+    pool.close(); model.close()
+
+
+# ---------------------------------------------------------------- boundary behaviour on the device
+def test_miss_is_reported_and_nothing_is_enqueued():
+    B, rt = _runtime()
+    shape = small_bf16_shape()
+    batch = _tiny_batch(shape, 80, [100, 100], [4, 4], [8, 8])
+    w, model, pool, db = _setup(shape, 25, batch)
+    status = np.zeros(2, dtype=np.int32)
+    n0 = model.launch_count()
+    # users are ALLOCATED but never pre-inferred: rank must refuse
+    assert pool.rank(db, per_user_status=status, ok=(B.E_MISS,)) is None
+    assert list(status) == [B.TIER_ALLOCATED, B.TIER_ALLOCATED]
+    assert model.launch_count() == n0
+    pool.preinfer(db)
+    unknown = synth.Batch(np.array([0, 99], np.uint64), batch.prefix_ids, batch.prefix_off, batch.short_ids, batch.short_off,
+                          batch.cand_ids, batch.cand_off)
+    assert pool.rank(rt.DeviceBatch(unknown, model.device), per_user_status=status, ok=(B.E_MISS,)) is None
+    assert list(status) == [B.TIER_HBM, B.TIER_MISS]
+    # wrong prefix length at pre-infer
+    pool.alloc(7, 50)
+    bad = synth.Batch(np.array([7], np.uint64), batch.prefix_ids[:60], np.array([0, 60], np.int32), batch.short_ids[:0],
+                      np.array([0, 0], np.int32), batch.cand_ids[:0], np.array([0, 0], np.int32))
+    assert pool.preinfer(rt.DeviceBatch(bad, model.device), ok=(B.E_INVALID,)) == B.E_INVALID
+    assert pool.stats()["misses"] >= 1
+    pool.close(); model.close()
+
+
+def test_spill_and_reload_round_trip_is_bit_exact():
+    B, rt = _runtime()
+    shape = small_bf16_shape()
+    batch = _tiny_batch(shape, 81, [300, 640], [9, 3], [60, 70])
+    w, model, pool, db = _setup(shape, 26, batch, hbm_pages=20, host_pages=20)
+    pool.preinfer(db)
+    ref_scores = pool.rank(db).cpu().numpy().copy()
+    kv0 = [tuple(t.clone() for t in pool.read_kv(u, p)) for u, p in zip(batch.users, (300, 640))]
+    side = torch.cuda.Stream()
+    for u in batch.users:
+        pool.evict(u, True, side)
+    assert [pool.lookup(u)[0] for u in batch.users] == [B.TIER_HOST, B.TIER_HOST]
+    assert pool.stats()["pages_free"] == 20
+    assert pool.rank(db, ok=(B.E_MISS,)) is None
+    # scribble over the slab so a reload has to bring the bytes back
+    side.synchronize()
+    pool.slab.fill_(0x7f)
+    for u in batch.users:
+        code, ev = pool.reload(u, side)
+        assert code == B.OK
+        code2, ev2 = pool.reload(u, side)            # single-flight / idempotent
+        assert code2 == B.OK
+    st = pool.stats()
+    assert st["reloads"] == 2 and st["spills"] == 2 and st["reload_bytes"] == st["spill_bytes"]
+    scores = pool.rank(db).cpu().numpy()             # rank orders itself behind the reload events
+    torch.cuda.synchronize()
+    assert np.array_equal(scores.view(np.uint32), ref_scores.view(np.uint32))
+    for (k0, v0), u, p in zip(kv0, batch.users, (300, 640)):
+        k1, v1 = pool.read_kv(u, p)
+        assert torch.equal(k0, k1) and torch.equal(v0, v1)
+    pool.close(); model.close()
