@@ -135,6 +135,15 @@ int32_t relaygr_workspace_bytes(const relaygr_ctx *ctx, int64_t max_rows, int64_
                                 size_t *out_bytes);
 int32_t relaygr_set_workspace(relaygr_ctx *ctx, void *dev, size_t bytes);
 
+/*
+ * Kernels never trap, and their internal waits are bounded: a kernel that meets an
+ * impossible state (a wait that ran out) records a code in a status word at the start
+ * of the workspace and the kernels after it return early, leaving results undefined.
+ * This call SYNCHRONISES `stream`, then copies the word to *out (0 = healthy).
+ * relaygr_set_workspace clears the word (synchronously).
+ */
+int32_t relaygr_device_status(relaygr_ctx *ctx, void *stream, int32_t *out);
+
 /* ---- paged prefix-KV pool (Section 3.3 sliding window, Section 3.4 DRAM tier) ---------------- */
 
 /*

@@ -59,6 +59,7 @@ SIGNATURES = {
     "relaygr_last_error": (C.c_char_p, []),
     "relaygr_workspace_bytes": (_I32, [_P, _I64, _I64, _I64, C.POINTER(_SZ)]),
     "relaygr_set_workspace": (_I32, [_P, _P, _SZ]),
+    "relaygr_device_status": (_I32, [_P, _P, C.POINTER(_I32)]),
     "relaygr_kv_page_bytes": (_I32, [_P, C.POINTER(_SZ)]),
     "relaygr_kv_pool_create": (_I32, [_P, _P, _SZ, _P, _SZ, C.POINTER(_P)]),
     "relaygr_kv_pool_destroy": (_I32, [_P]),
@@ -151,6 +152,12 @@ def relaygr_workspace_bytes(ctx, max_rows, max_users, max_pages) -> int:
 
 def relaygr_set_workspace(ctx, dev, nbytes):
     _check(lib().relaygr_set_workspace(ctx, _ptr(dev), nbytes))
+
+
+def relaygr_device_status(ctx, stream=None) -> int:
+    out = _I32()
+    _check(lib().relaygr_device_status(ctx, stream, C.byref(out)))
+    return out.value
 
 
 def relaygr_kv_page_bytes(ctx) -> int:

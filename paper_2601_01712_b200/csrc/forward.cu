@@ -4,6 +4,7 @@
 #include <cstring>
 
 #include "kernels.cuh"
+#include "tc_common.cuh"
 
 namespace relaygr {
 
@@ -32,6 +33,40 @@ int Forward::init_device(int dev, std::string &err)
         e = cudaEventCreateWithFlags(&slot_event[i], cudaEventDisableTiming);
         if (e != cudaSuccess) { err = cuda_msg("cudaEventCreate", e); return RELAYGR_E_CUDA; }
     }
+    if (cfg.dtype == RELAYGR_DTYPE_BF16) {
+        const uint64_t d = (uint64_t)cfg.d_model, F = (uint64_t)cfg.d_ff;
+        wmaps.resize((size_t)cfg.n_layers);
+        for (int l = 0; l < cfg.n_layers; ++l) {
+            const __nv_bfloat16 *wq = (const __nv_bfloat16 *)w.w_qkv + (size_t)l * 3 * d * d;
+            int rc = make_tmap_2d_bf16(&wmaps[(size_t)l].qkv, wq, 3 * d, d, d, 128, 64);
+            rc |= make_tmap_2d_bf16(&wmaps[(size_t)l].kv, wq + d * d, 2 * d, d, d, 128, 64);
+            rc |= make_tmap_2d_bf16(&wmaps[(size_t)l].wo, (const __nv_bfloat16 *)w.w_o + (size_t)l * d * d, d, d, d, 128, 64);
+            rc |= make_tmap_2d_bf16(&wmaps[(size_t)l].w1, (const __nv_bfloat16 *)w.w1 + (size_t)l * F * d, F, d, d, 128, 64);
+            rc |= make_tmap_2d_bf16(&wmaps[(size_t)l].w2, (const __nv_bfloat16 *)w.w2 + (size_t)l * d * F, d, F, F, 128, 64);
+            if (rc != 0) { err = "tensor-map encoding of the weights failed (pointers must be 16-byte aligned)"; return RELAYGR_E_CUDA; }
+        }
+    }
+    return RELAYGR_OK;
+}
+
+int Forward::set_workspace(void *dev, size_t bytes, std::string &err)
+{
+    ws = (char *)dev;
+    ws_bytes = dev ? bytes : 0;
+    if (ws && ws_bytes >= 1024) {
+        cudaError_t e = cudaMemset(ws, 0, 1024);      // the status word starts clean
+        if (e != cudaSuccess) { err = cuda_msg("cudaMemset (workspace status)", e); return RELAYGR_E_CUDA; }
+    }
+    return RELAYGR_OK;
+}
+
+int Forward::device_status(cudaStream_t stream, int32_t *out, std::string &err)
+{
+    *out = 0;
+    if (!ws) return RELAYGR_OK;
+    cudaError_t e = cudaStreamSynchronize(stream);
+    if (e == cudaSuccess) e = cudaMemcpy(out, ws, 4, cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) { err = cuda_msg("device status read", e); return RELAYGR_E_CUDA; }
     return RELAYGR_OK;
 }
 
@@ -42,6 +77,7 @@ WorkspaceLayout Forward::layout(int64_t rows, int64_t users, int64_t pages) cons
     const size_t r = (size_t)rows + 128;    // slack so that 128-row tiles may read past the last row
     size_t at = 0;
     auto take = [&](size_t bytes) { const size_t o = at; at = align_up(at + bytes, 1024); return o; };
+    l.status = take(1024);
     l.x = take(r * d * 4);
     l.a = take(r * d * es);
     l.q = take(r * d * es);
@@ -153,6 +189,22 @@ int Forward::run_t(const CallDesc &call, float *scores, cudaStream_t stream, std
     cudaError_t e = cudaSuccess;
     auto ck = [&](const char *what) -> bool { if (e != cudaSuccess) { err = cuda_msg(what, e); return false; } return true; };
 
+    // bf16 model: GEMMs and attention run on the tensor cores; per-call tensor maps of the activations
+    constexpr bool kTensor = sizeof(T) == 2;
+    int *d_status = reinterpret_cast<int *>(ws + lay.status);
+    CUtensorMap tm_a, tm_att, tm_hid;
+    if (kTensor) {
+        int trc = make_tmap_2d_bf16(&tm_a, a, (uint64_t)R, (uint64_t)d, (uint64_t)d, 128, 64);
+        trc |= make_tmap_2d_bf16(&tm_att, att, (uint64_t)R, (uint64_t)d, (uint64_t)d, 128, 64);
+        trc |= make_tmap_2d_bf16(&tm_hid, hid, (uint64_t)R, (uint64_t)F, (uint64_t)F, 128, 64);
+        if (trc != 0) { err = "tensor-map encoding of the activations failed"; return RELAYGR_E_CUDA; }
+    }
+    auto gemm = [&](const T *A, const CUtensorMap &tmA, const T *W, const CUtensorMap *tmW, int N, int K, const Epilogue &ep) {
+        if constexpr (kTensor) return launch_gemm_tc(tmA, *tmW, R, N, K, ep, d_status, stream, &launches);
+        else return launch_gemm_simt<T>(A, W, R, N, K, ep, stream, &launches);
+    };
+    const LayerMaps *lm = nullptr;
+
     for (int l = 0; l < L; ++l) {
         const float *g1 = w.ln1_g + (size_t)l * d, *b1n = w.ln1_b + (size_t)l * d;
         if (l == 0) e = launch_gather_ln<T>((const T *)w.emb, cfg.vocab, d, src, R, g1, b1n, cfg.ln_eps, x, a, stream, &launches);
@@ -174,7 +226,8 @@ int Forward::run_t(const CallDesc &call, float *scores, cudaStream_t stream, std
         }
         if (preinfer) ep.paged = paged;
         const T *Wqkv = (const T *)w.w_qkv + ((size_t)l * 3 * d + ep.col0) * d;
-        e = launch_gemm_simt<T>(a, Wqkv, R, 3 * d - ep.col0, d, ep, stream, &launches);
+        lm = kTensor ? &wmaps[(size_t)l] : nullptr;
+        e = gemm(a, tm_a, Wqkv, lm ? (kv_only ? &lm->kv : &lm->qkv) : nullptr, 3 * d - ep.col0, d, ep);
         if (!ck("QKV projection")) return RELAYGR_E_CUDA;
         if (kv_only) break;
 
@@ -183,7 +236,7 @@ int Forward::run_t(const CallDesc &call, float *scores, cudaStream_t stream, std
 
         Epilogue eo{};
         eo.mode = EPI_RESID; eo.bias = w.b_o ? w.b_o + (size_t)l * d : nullptr; eo.resid = x; eo.out_f32 = x;
-        e = launch_gemm_simt<T>(att, (const T *)w.w_o + (size_t)l * d * d, R, d, d, eo, stream, &launches);
+        e = gemm(att, tm_att, (const T *)w.w_o + (size_t)l * d * d, lm ? &lm->wo : nullptr, d, d, eo);
         if (!ck("output projection")) return RELAYGR_E_CUDA;
 
         e = launch_layernorm<T>(x, d, R, w.ln2_g + (size_t)l * d, w.ln2_b + (size_t)l * d, cfg.ln_eps, a, stream, &launches);
@@ -191,12 +244,12 @@ int Forward::run_t(const CallDesc &call, float *scores, cudaStream_t stream, std
 
         Epilogue e1{};
         e1.mode = EPI_STORE; e1.silu = 1; e1.bias = w.b1 ? w.b1 + (size_t)l * F : nullptr; e1.out = hid;
-        e = launch_gemm_simt<T>(a, (const T *)w.w1 + (size_t)l * F * d, R, F, d, e1, stream, &launches);
+        e = gemm(a, tm_a, (const T *)w.w1 + (size_t)l * F * d, lm ? &lm->w1 : nullptr, F, d, e1);
         if (!ck("FFN 1")) return RELAYGR_E_CUDA;
 
         Epilogue e2{};
         e2.mode = EPI_RESID; e2.bias = w.b2 ? w.b2 + (size_t)l * d : nullptr; e2.resid = x; e2.out_f32 = x;
-        e = launch_gemm_simt<T>(hid, (const T *)w.w2 + (size_t)l * d * F, R, d, F, e2, stream, &launches);
+        e = gemm(hid, tm_hid, (const T *)w.w2 + (size_t)l * d * F, lm ? &lm->w2 : nullptr, d, F, e2);
         if (!ck("FFN 2")) return RELAYGR_E_CUDA;
     }
 

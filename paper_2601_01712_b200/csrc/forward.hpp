@@ -6,6 +6,7 @@
 #include <string>
 #include <vector>
 
+#include <cuda.h>
 #include <cuda_runtime.h>
 
 #include "../../include/relaygr.h"
@@ -28,7 +29,7 @@ struct CallDesc {
 };
 
 struct WorkspaceLayout {
-    size_t x, a, q, k, v, att, hid, partial, meta, total;
+    size_t status, x, a, q, k, v, att, hid, partial, meta, total;
     size_t meta_bytes, partial_bytes;
 };
 
@@ -50,6 +51,10 @@ struct Forward {
     int device = 0;
     int n_sms = 148;
 
+    // tensor maps of the weights (bf16 model), one set per layer
+    struct LayerMaps { CUtensorMap qkv, kv, wo, w1, w2; };
+    std::vector<LayerMaps> wmaps;
+
     // pinned staging ring for the per-call metadata
     static constexpr int kSlots = 4;
     static constexpr size_t kSlotBytes = 2u << 20;
@@ -64,6 +69,8 @@ struct Forward {
     int check_capacity(const CallDesc &call, std::string &err) const;
     int run(const CallDesc &call, float *scores, cudaStream_t stream, std::string &err);
     int gather(const int32_t *ids, int64_t n, void *out, cudaStream_t stream, std::string &err);
+    int set_workspace(void *dev, size_t bytes, std::string &err);
+    int device_status(cudaStream_t stream, int32_t *out, std::string &err);
 
     size_t esize() const { return cfg.dtype == RELAYGR_DTYPE_F32 ? 4 : 2; }
     static constexpr int64_t kMaxSplitTiles = 1536;   // capacity of the split-KV partial buffer, in 128-row tiles

@@ -2,6 +2,8 @@
 // cudaError_t of the launch and adds the number of kernels it launched to *launches.
 #pragma once
 
+#include <cuda.h>
+
 #include "internal.cuh"
 
 namespace relaygr {
@@ -41,5 +43,13 @@ template <typename T>
 cudaError_t launch_attention_simt(const T *q, const T *k_lin, const T *v_lin, PagedKV paged, const SeqDesc *seqs,
                                   const int32_t *row_off, int n_users, int64_t n_rows, int n_heads, int d_head,
                                   T *out, cudaStream_t stream, int64_t *launches);
+
+// ---- tensor-core kernels (the bf16 model) -------------------------------------------------------------
+
+// C[m, n] = sum_k A[m, k] W[n, k] on tcgen05; tmA covers A [M, K] with a 128-row box, tmB covers W [N, K]
+// with a 128-row box, both 64 columns wide with the 128-byte swizzle.  N % 128 == 0, K % 64 == 0.
+// err is a device status word: kernels record a code there instead of hanging or trapping.
+cudaError_t launch_gemm_tc(const CUtensorMap &tmA, const CUtensorMap &tmB, int64_t M, int N, int K, const Epilogue &epi,
+                           int *err, cudaStream_t stream, int64_t *launches);
 
 }  // namespace relaygr

@@ -125,9 +125,16 @@ int32_t relaygr_set_workspace(relaygr_ctx *ctx, void *dev, size_t bytes)
 {
     if (!ctx) return fail(RELAYGR_E_INVALID, "ctx is NULL");
     if (((uintptr_t)dev & 255) != 0) return fail(RELAYGR_E_INVALID, "workspace must be 256-byte aligned");
-    ctx->fwd.ws = (char *)dev;
-    ctx->fwd.ws_bytes = dev ? bytes : 0;
-    return RELAYGR_OK;
+    if (ctx->host_only) return RELAYGR_OK;
+    return ctx->fwd.set_workspace(dev, bytes, g_err);
+}
+
+int32_t relaygr_device_status(relaygr_ctx *ctx, void *stream, int32_t *out)
+{
+    if (!ctx || !out) return fail(RELAYGR_E_INVALID, "bad argument");
+    *out = 0;
+    if (ctx->host_only) return RELAYGR_OK;
+    return ctx->fwd.device_status((cudaStream_t)stream, out, g_err);
 }
 
 int32_t relaygr_launch_count(const relaygr_ctx *ctx, int64_t *out)

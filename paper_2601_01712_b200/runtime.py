@@ -73,6 +73,10 @@ class Model:
                             scores.data_ptr(), _stream_ptr(stream))
         return scores
 
+    def device_status(self, stream=None) -> int:
+        """Synchronises the stream and returns the kernels' status word (0 = healthy)."""
+        return B.relaygr_device_status(self.ctx, _stream_ptr(stream))
+
     def launch_count(self) -> int:
         return B.relaygr_launch_count(self.ctx)
 

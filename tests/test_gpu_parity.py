@@ -63,6 +63,7 @@ def test_config1_fp32_preinfer_rank_full():
     # the paper's relation: rank on cache ~= full inference
     assert np.max(np.abs(scores.cpu().numpy() - full.cpu().numpy())) <= TOL_F32
     assert model.launch_count() > 0
+    assert model.device_status() == 0
     pool.close(); model.close()
 
 
@@ -111,6 +112,7 @@ def test_jagged_bf16_matches_checker(case):
     want = oracle_scores(om, batch)
     assert max_abs_err(scores.cpu().numpy(), batch, want) <= TOL_BF16
     assert max_abs_err(full.cpu().numpy(), batch, want) <= TOL_BF16
+    assert model.device_status() == 0
     pool.close(); model.close()
 
 
@@ -132,7 +134,8 @@ def test_shuffled_page_table_changes_nothing():
                 assert np.array_equal(pool.pages(batch.users[i]), ids[i])
         kv = [tuple(t.view(torch.int16).cpu().numpy() for t in pool.read_kv(batch.users[i], p[i])) for i in range(3)]
         res.append((scores.cpu().numpy().copy(), kv))
-        pool.close(); model.close()
+        assert model.device_status() == 0
+    pool.close(); model.close()
     assert np.array_equal(res[0][0].view(np.uint32), res[1][0].view(np.uint32))
     for a, b in zip(res[0][1], res[1][1]):
         assert np.array_equal(a[0], b[0]) and np.array_equal(a[1], b[1])
@@ -156,6 +159,7 @@ def test_preinfer_is_deterministic_and_rank_leaves_pages_untouched():
     pool.preinfer(db)
     torch.cuda.synchronize()
     assert torch.equal(before, pool.slab)
+    assert model.device_status() == 0
     pool.close(); model.close()
 
 
@@ -172,6 +176,7 @@ def test_batch_equals_single_user_calls_and_candidate_independence():
                       batch.cand_ids[200 + 10:200 + 30], np.array([0, 20], np.int32))
     s1 = pool.rank(rt.DeviceBatch(one, model.device)).cpu().numpy()
     assert np.max(np.abs(s1 - scores[200 + 10:200 + 30])) <= 1e-5
+    assert model.device_status() == 0
     pool.close(); model.close()
 
 
@@ -198,6 +203,7 @@ def test_miss_is_reported_and_nothing_is_enqueued():
                       np.array([0, 0], np.int32), batch.cand_ids[:0], np.array([0, 0], np.int32))
     assert pool.preinfer(rt.DeviceBatch(bad, model.device), ok=(B.E_INVALID,)) == B.E_INVALID
     assert pool.stats()["misses"] >= 1
+    assert model.device_status() == 0
     pool.close(); model.close()
 
 
@@ -231,4 +237,5 @@ def test_spill_and_reload_round_trip_is_bit_exact():
     for (k0, v0), u, p in zip(kv0, batch.users, (300, 640)):
         k1, v1 = pool.read_kv(u, p)
         assert torch.equal(k0, k1) and torch.equal(v0, v1)
+    assert model.device_status() == 0
     pool.close(); model.close()
