@@ -1,0 +1,396 @@
+// Flash-style attention on tcgen05 for the bf16 model (d_head = 64), serving all three passes:
+// pre-infer (causal over the user's own pages), rank on cache (prefix pages through the page
+// table + short-term rows + the candidate's own row) and full inference (linear K/V rows).
+//
+// One CTA = one work item: a 128-row query tile of one head of one user against a range of
+// that user's 128-key blocks.  Per block:  S = Q K^T  (tcgen05.mma, M=128 N=128 K=64, operands in
+// shared memory, S in TMEM) -> online softmax by 128 threads, one row each, P written back to
+// TMEM as bf16 -> O += P V (tcgen05.mma, M=128 N=64 K=128, A = P from TMEM, B = V in shared
+// memory, MN-major, O accumulated in TMEM).  The running maximum is only raised (and O rescaled
+// in TMEM) when it grows by more than 2^8, which keeps every exponent in range and makes the
+// rescale rare.  K/V tiles are two 64-row TMA boxes each: 64-token pages of the pool addressed
+// through the page table, or rows of the call's transient K/V buffers.
+//
+// Warp roles (192 threads): warp 0 = TMA producer, warp 1 = TMEM owner + MMA issuer,
+// warps 2-5 = softmax / correction / epilogue (TMEM lane quadrant = warp index % 4).
+// Two CTAs per SM: one CTA's softmax overlaps the other's MMAs.
+#include "kernels.cuh"
+#include "tc_common.cuh"
+
+namespace relaygr {
+
+namespace {
+
+constexpr int kQTile = 128, kKeys = 128, kDh = 64;
+constexpr int kQBytes = kQTile * kDh * 2;           // 16 KB
+constexpr int kKVBytes = kKeys * kDh * 2;           // 16 KB per K or V tile (two 8 KB boxes)
+constexpr int kStagesKV = 2;
+constexpr int kSmemBytes = kQBytes + 2 * kStagesKV * kKVBytes + 1024 + 256;
+constexpr uint32_t kTmemCols = 256;                 // S: 0..127, P: 128..191, O: 192..255
+constexpr uint32_t kColS = 0, kColP = 128, kColO = 192;
+constexpr float kRescaleThreshold = 8.f;            // in log2 units
+
+struct Bars {
+    uint64_t q_full;
+    uint64_t k_full[kStagesKV], k_empty[kStagesKV], v_full[kStagesKV], v_empty[kStagesKV];
+    uint64_t s_full, s_free, p_full, pv_done;
+    uint32_t tmem_slot;
+    int abort_flag;
+};
+
+__device__ __forceinline__ float ex2(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+__global__ void __launch_bounds__(192, 2)
+attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmKlin,
+                    const __grid_constant__ CUtensorMap tmVlin, const __grid_constant__ CUtensorMap tmPool,
+                    const AttnItem *__restrict__ items, const SeqDesc *__restrict__ seqs, const int32_t *__restrict__ pt,
+                    int n_layers, int layer, int d_model, const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restrict__ k_lin,
+                    const __nv_bfloat16 *__restrict__ v_lin, __nv_bfloat16 *__restrict__ out, float *__restrict__ partial, int *err)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint8_t *sQ = smem;
+    uint8_t *sK = smem + kQBytes;
+    uint8_t *sV = sK + kStagesKV * kKVBytes;
+    Bars *bars = reinterpret_cast<Bars *>(sV + kStagesKV * kKVBytes);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const AttnItem it = items[blockIdx.x];
+    const SeqDesc sd = seqs[it.seq];
+    const int nb = it.blk1 - it.blk0;
+    const int n_paged_blocks = (sd.n_paged + kKeys - 1) / kKeys;
+
+    if (threadIdx.x == 0) bars->abort_flag = *reinterpret_cast<volatile int *>(err);
+    __syncthreads();
+    if (bars->abort_flag != 0) return;
+
+    if (threadIdx.x == 0) {
+        tc::mbar_init(&bars->q_full, 1);
+        for (int s = 0; s < kStagesKV; ++s) {
+            tc::mbar_init(&bars->k_full[s], 1); tc::mbar_init(&bars->k_empty[s], 1);
+            tc::mbar_init(&bars->v_full[s], 1); tc::mbar_init(&bars->v_empty[s], 1);
+        }
+        tc::mbar_init(&bars->s_full, 1);
+        tc::mbar_init(&bars->s_free, 128);
+        tc::mbar_init(&bars->p_full, 128);
+        tc::mbar_init(&bars->pv_done, 1);
+        tc::fence_mbar_init();
+        tc::tma_prefetch_desc(&tmQ); tc::tma_prefetch_desc(&tmKlin); tc::tma_prefetch_desc(&tmVlin); tc::tma_prefetch_desc(&tmPool);
+    }
+    if (warp == 1) {
+        tc::tmem_alloc(&bars->tmem_slot, kTmemCols);
+        tc::tmem_relinquish();
+    }
+    tc::tc_fence_before();
+    __syncthreads();
+    tc::tc_fence_after();
+    const uint32_t tmem_base = bars->tmem_slot;
+
+    if (warp == 0) {
+        // ---------------------------------------------------------------- TMA producer
+        if (lane == 0) {
+            tc::mbar_expect_tx(&bars->q_full, kQBytes);
+            tc::tma_load_2d(sQ, &tmQ, it.head * kDh, sd.q_row0 + it.q0, &bars->q_full);
+            for (int j = 0; j < nb; ++j) {
+                const int b = it.blk0 + j;
+                const int s = j % kStagesKV;
+                const uint32_t par = ((j / kStagesKV) & 1) ^ 1;
+                const bool paged = b < n_paged_blocks;
+                int y0, y1;              // first rows of the two 64-key halves (K); V rows follow from them
+                int vy0, vy1;
+                const CUtensorMap *mk, *mv;
+                if (paged) {
+                    const int p0 = pt[sd.pt_base + 2 * b];
+                    const bool two = (2 * b + 1) * 64 < sd.n_paged;
+                    const int p1 = two ? pt[sd.pt_base + 2 * b + 1] : p0;      // absent half: re-read the first page (masked later)
+                    y0 = ((p0 * n_layers + layer) * 2) * 64; y1 = ((p1 * n_layers + layer) * 2) * 64;
+                    vy0 = y0 + 64; vy1 = y1 + 64;
+                    mk = &tmPool; mv = &tmPool;
+                } else {
+                    const int r = sd.lin_row0 + (b - n_paged_blocks) * kKeys;
+                    y0 = r; y1 = r + 64; vy0 = y0; vy1 = y1;
+                    mk = &tmKlin; mv = &tmVlin;
+                }
+                if (!tc::mbar_wait(&bars->k_empty[s], par, err)) break;
+                tc::mbar_expect_tx(&bars->k_full[s], kKVBytes);
+                tc::tma_load_2d(sK + s * kKVBytes, mk, it.head * kDh, y0, &bars->k_full[s]);
+                tc::tma_load_2d(sK + s * kKVBytes + kKVBytes / 2, mk, it.head * kDh, y1, &bars->k_full[s]);
+                if (!tc::mbar_wait(&bars->v_empty[s], par, err)) break;
+                tc::mbar_expect_tx(&bars->v_full[s], kKVBytes);
+                tc::tma_load_2d(sV + s * kKVBytes, mv, it.head * kDh, vy0, &bars->v_full[s]);
+                tc::tma_load_2d(sV + s * kKVBytes + kKVBytes / 2, mv, it.head * kDh, vy1, &bars->v_full[s]);
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------------------------------------------------------- MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc_qk = tc::make_idesc(128, 128, 0, 0);     // Q, K both K-major
+            constexpr uint32_t idesc_pv = tc::make_idesc(128, 64, 0, 1);      // P from TMEM, V MN-major
+            const uint64_t qdesc = tc::smem_desc_sw128(tc::smem_u32(sQ));
+            bool ok = tc::mbar_wait(&bars->q_full, 0, err);
+            auto issue_qk = [&](int j) {
+                const int s = j % kStagesKV;
+                if (!tc::mbar_wait(&bars->k_full[s], (j / kStagesKV) & 1, err)) return false;
+                if (j > 0 && !tc::mbar_wait(&bars->s_free, (j - 1) & 1, err)) return false;
+                tc::tc_fence_after();
+                const uint64_t kdesc = tc::smem_desc_sw128(tc::smem_u32(sK + s * kKVBytes));
+#pragma unroll
+                for (int k = 0; k < kDh / 16; ++k) tc::mma_ss(tmem_base + kColS, qdesc + 2 * k, kdesc + 2 * k, idesc_qk, k != 0);
+                tc::mma_commit(&bars->s_full);
+                tc::mma_commit(&bars->k_empty[s]);
+                return true;
+            };
+            if (ok && nb > 0) ok = issue_qk(0);
+            for (int j = 0; j < nb && ok; ++j) {
+                if (j + 1 < nb) { ok = issue_qk(j + 1); if (!ok) break; }
+                const int s = j % kStagesKV;
+                if (!tc::mbar_wait(&bars->p_full, j & 1, err)) break;
+                if (!tc::mbar_wait(&bars->v_full[s], (j / kStagesKV) & 1, err)) break;
+                tc::tc_fence_after();
+                const uint64_t vdesc = tc::smem_desc_sw128(tc::smem_u32(sV + s * kKVBytes));
+#pragma unroll
+                for (int k = 0; k < kKeys / 16; ++k)      // 16 keys per instruction: 8 TMEM columns of P, 2048 bytes of V
+                    tc::mma_ts(tmem_base + kColO, tmem_base + kColP + 8 * k, vdesc + 128 * k, idesc_pv, (j | k) != 0);
+                tc::mma_commit(&bars->pv_done);
+                tc::mma_commit(&bars->v_empty[s]);
+            }
+        }
+    } else {
+        // ---------------------------------------------------------------- softmax / correction / epilogue
+        const int quad = warp & 3;
+        const int r = quad * 32 + lane;                      // row of the tile this thread owns
+        const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
+        const int tpos = sd.q_pos0 + it.q0 + r;              // sequence position of the row
+        const bool is_cand = tpos >= sd.causal_end;
+        const int lim = is_cand ? sd.causal_end - 1 : tpos;  // last visible key position
+        const int tile_min_lim = (sd.q_pos0 + it.q0 >= sd.causal_end) ? sd.causal_end - 1 : sd.q_pos0 + it.q0;
+        const float c = 0.125f * 1.4426950408889634f;        // 1/sqrt(64) * log2(e)
+        float m = -INFINITY, l = 0.f;
+        bool ok = true;
+
+        for (int j = 0; j < nb && ok; ++j) {
+            const int b = it.blk0 + j;
+            const bool paged = b < n_paged_blocks;
+            const int kidx0 = paged ? b * kKeys : (b - n_paged_blocks) * kKeys;        // index of the block's first key in its source
+            const int kpos0 = paged ? kidx0 : sd.lin_pos0 + kidx0;                     // its sequence position
+            const int n_valid = min(kKeys, (paged ? sd.n_paged : sd.n_lin) - kidx0);
+            const bool need_mask = (n_valid < kKeys) || (kpos0 + kKeys - 1 > tile_min_lim);
+            const int jmax = min(n_valid, lim - kpos0 + 1);  // keys jj < jmax of this block are visible to this row
+
+            ok = __all_sync(0xffffffffu, tc::mbar_wait(&bars->s_full, j & 1, err));
+            if (!ok) break;
+            tc::tc_fence_after();
+
+            // pass 1: row maximum
+            float mx = -INFINITY;
+#pragma unroll 1
+            for (int cc = 0; cc < kKeys; cc += 32) {
+                uint32_t sv[32];
+                tc::tmem_ld32(lane_addr + kColS + cc, sv);
+                tc::tmem_ld_wait();
+                if (need_mask) {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) mx = fmaxf(mx, (cc + i < jmax) ? __uint_as_float(sv[i]) : -INFINITY);
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(sv[i]));
+                }
+            }
+            // raise the running maximum only when it grows by more than the threshold
+            float alpha = 1.f;
+            bool raise = (mx - m) * c > kRescaleThreshold;          // false when mx == -inf; true on the first visible key
+            if (raise) {
+                alpha = (m == -INFINITY) ? 0.f : ex2((m - mx) * c);
+                m = mx;
+            }
+            const float mc = (m == -INFINITY) ? 0.f : m * c;
+
+            // P(j) overwrites P(j-1) and the correction touches O: both need PV(j-1) complete
+            if (j > 0) {
+                ok = __all_sync(0xffffffffu, tc::mbar_wait(&bars->pv_done, (j - 1) & 1, err));
+                if (!ok) break;
+                tc::tc_fence_after();
+                if (__any_sync(0xffffffffu, raise)) {
+#pragma unroll 1
+                    for (int cc = 0; cc < kDh; cc += 16) {
+                        uint32_t ov[16];
+                        tc::tmem_ld16(lane_addr + kColO + cc, ov);
+                        tc::tmem_ld_wait();
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) ov[i] = __float_as_uint(__uint_as_float(ov[i]) * alpha);
+                        tc::tmem_st16(lane_addr + kColO + cc, ov);
+                    }
+                }
+            }
+            l *= alpha;
+
+            // pass 2: p = 2^(s c - m c), row sum, bf16 P into TMEM
+            float rs = 0.f;
+#pragma unroll 1
+            for (int cc = 0; cc < kKeys; cc += 32) {
+                uint32_t sv[32];
+                tc::tmem_ld32(lane_addr + kColS + cc, sv);
+                tc::tmem_ld_wait();
+                float p[32];
+                if (need_mask) {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) p[i] = (cc + i < jmax) ? ex2(fmaf(__uint_as_float(sv[i]), c, -mc)) : 0.f;
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) p[i] = ex2(fmaf(__uint_as_float(sv[i]), c, -mc));
+                }
+                uint32_t pk[16];
+#pragma unroll
+                for (int i = 0; i < 16; ++i) { rs += p[2 * i] + p[2 * i + 1]; pk[i] = tc::pack_bf16(p[2 * i], p[2 * i + 1]); }
+                tc::tmem_st16(lane_addr + kColP + cc / 2, pk);
+            }
+            l += rs;
+            tc::tc_fence_before();
+            tc::mbar_arrive(&bars->s_free);        // S(j) fully read: the next QK^T may overwrite it
+            tc::tmem_st_wait();
+            tc::tc_fence_before();
+            tc::mbar_arrive(&bars->p_full);        // P(j) (and any correction of O) is in TMEM
+        }
+
+        // ---- epilogue: O / l (plus the candidate's own key), or the split partial
+        if (ok && nb > 0) ok = __all_sync(0xffffffffu, tc::mbar_wait(&bars->pv_done, (nb - 1) & 1, err));
+        tc::tc_fence_after();
+        if (ok) {
+            float o[kDh];
+            if (nb > 0) {
+#pragma unroll
+                for (int cc = 0; cc < kDh; cc += 16) {
+                    uint32_t ov[16];
+                    tc::tmem_ld16(lane_addr + kColO + cc, ov);
+                    tc::tmem_ld_wait();
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) o[cc + i] = __uint_as_float(ov[i]);
+                }
+            } else {
+#pragma unroll
+                for (int i = 0; i < kDh; ++i) o[i] = 0.f;
+            }
+            const bool row_ok = r < it.n_q;
+            const int64_t row = (int64_t)sd.q_row0 + it.q0 + r;
+            if (row_ok && is_cand && it.with_self) {
+                // the candidate's own key / value row, folded into the running softmax on CUDA cores
+                const uint4 *qp = reinterpret_cast<const uint4 *>(q + row * d_model + it.head * kDh);
+                const uint4 *kp = reinterpret_cast<const uint4 *>(k_lin + row * d_model + it.head * kDh);
+                const uint4 *vp = reinterpret_cast<const uint4 *>(v_lin + row * d_model + it.head * kDh);
+                float dot = 0.f;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const uint4 a = qp[i], bq = kp[i];
+                    const __nv_bfloat162 *a2 = reinterpret_cast<const __nv_bfloat162 *>(&a);
+                    const __nv_bfloat162 *b2 = reinterpret_cast<const __nv_bfloat162 *>(&bq);
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float2 fa = __bfloat1622float2(a2[e]), fb = __bfloat1622float2(b2[e]);
+                        dot = fmaf(fa.x, fb.x, dot); dot = fmaf(fa.y, fb.y, dot);
+                    }
+                }
+                const float mn = fmaxf(m, dot);
+                const float al = (m == -INFINITY) ? 0.f : ex2((m - mn) * c);
+                const float ps = ex2((dot - mn) * c);
+                l = l * al + ps;
+                m = mn;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const uint4 vv = vp[i];
+                    const __nv_bfloat162 *v2 = reinterpret_cast<const __nv_bfloat162 *>(&vv);
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float2 fv = __bfloat1622float2(v2[e]);
+                        o[i * 8 + 2 * e] = fmaf(o[i * 8 + 2 * e], al, ps * fv.x);
+                        o[i * 8 + 2 * e + 1] = fmaf(o[i * 8 + 2 * e + 1], al, ps * fv.y);
+                    }
+                }
+            }
+            if (row_ok) {
+                if (it.partial_slot < 0) {
+                    const float inv = 1.f / l;
+                    uint4 *dst = reinterpret_cast<uint4 *>(out + row * d_model + it.head * kDh);
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        uint4 w4;
+                        w4.x = tc::pack_bf16(o[8 * i] * inv, o[8 * i + 1] * inv);
+                        w4.y = tc::pack_bf16(o[8 * i + 2] * inv, o[8 * i + 3] * inv);
+                        w4.z = tc::pack_bf16(o[8 * i + 4] * inv, o[8 * i + 5] * inv);
+                        w4.w = tc::pack_bf16(o[8 * i + 6] * inv, o[8 * i + 7] * inv);
+                        dst[i] = w4;
+                    }
+                } else {
+                    float *dst = partial + ((size_t)it.partial_slot * kQTile + r) * (kDh + 2);
+                    dst[0] = m; dst[1] = l;
+#pragma unroll
+                    for (int i = 0; i < kDh; ++i) dst[2 + i] = o[i];
+                }
+            }
+        }
+    }
+    tc::tc_fence_before();
+    __syncthreads();
+    if (warp == 1) tc::tmem_dealloc(tmem_base, kTmemCols);
+}
+
+// Combine the (m, l, O) partials of a split work item:  O = sum_i 2^((m_i - M) c) O_i / sum_i 2^((m_i - M) c) l_i.
+__global__ void __launch_bounds__(128)
+attention_merge_kernel(const AttnMerge *__restrict__ merges, const SeqDesc *__restrict__ seqs, const float *__restrict__ partial,
+                       int d_model, __nv_bfloat16 *__restrict__ out)
+{
+    const AttnMerge mg = merges[blockIdx.x];
+    const int r = threadIdx.x;
+    if (r >= mg.n_q) return;
+    const float c = 0.125f * 1.4426950408889634f;
+    float M = -INFINITY;
+    for (int i = 0; i < mg.n_splits; ++i) M = fmaxf(M, partial[((size_t)(mg.slot0 + i) * kQTile + r) * (kDh + 2)]);
+    float o[kDh];
+#pragma unroll
+    for (int e = 0; e < kDh; ++e) o[e] = 0.f;
+    float l = 0.f;
+    for (int i = 0; i < mg.n_splits; ++i) {
+        const float *p = partial + ((size_t)(mg.slot0 + i) * kQTile + r) * (kDh + 2);
+        const float mi = p[0];
+        const float wgt = (mi == -INFINITY) ? 0.f : ex2((mi - M) * c);
+        l = fmaf(p[1], wgt, l);
+#pragma unroll
+        for (int e = 0; e < kDh; ++e) o[e] = fmaf(p[2 + e], wgt, o[e]);
+    }
+    const float inv = 1.f / l;
+    const int64_t row = (int64_t)seqs[mg.seq].q_row0 + mg.q0 + r;
+    __nv_bfloat16 *dst = out + row * d_model + mg.head * kDh;
+#pragma unroll
+    for (int e = 0; e < kDh; e += 2) *reinterpret_cast<uint32_t *>(dst + e) = tc::pack_bf16(o[e] * inv, o[e + 1] * inv);
+}
+
+}  // namespace
+
+cudaError_t launch_attention_tc(const CUtensorMap &tmQ, const CUtensorMap &tmK, const CUtensorMap &tmV, const CUtensorMap &tmPool,
+                                const AttnItem *items, int n_items, const AttnMerge *merges, int n_merges, const SeqDesc *seqs,
+                                const int32_t *pt, int n_layers, int layer, int d_model, const __nv_bfloat16 *q,
+                                const __nv_bfloat16 *k_lin, const __nv_bfloat16 *v_lin, __nv_bfloat16 *out, float *partial,
+                                int *err, cudaStream_t stream, int64_t *launches)
+{
+    if (n_items == 0) return cudaSuccess;
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    attention_tc_kernel<<<n_items, 192, kSmemBytes, stream>>>(tmQ, tmK, tmV, tmPool, items, seqs, pt, n_layers, layer, d_model, q,
+                                                              k_lin, v_lin, out, partial, err);
+    *launches += 1;
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess || n_merges == 0) return e;
+    attention_merge_kernel<<<n_merges, 128, 0, stream>>>(merges, seqs, partial, d_model, out);
+    *launches += 1;
+    return cudaGetLastError();
+}
+
+}  // namespace relaygr

@@ -88,7 +88,7 @@ WorkspaceLayout Forward::layout(int64_t rows, int64_t users, int64_t pages) cons
     l.partial_bytes = (size_t)kMaxSplitTiles * 128 * (size_t)(cfg.d_head + 2) * 4;
     l.partial = take(l.partial_bytes);
     const size_t n_items = (size_t)cfg.n_heads * ((size_t)rows / 128 + (size_t)users + 1) + 2 * (size_t)kMaxSplitTiles;
-    l.meta_bytes = 4 * (((size_t)users + 1) * 5 + (size_t)users * (sizeof(SeqDesc) / 4) + (size_t)pages + n_items * (sizeof(AttnWork) / 4) + 64);
+    l.meta_bytes = 4 * (((size_t)users + 1) * 5 + (size_t)users * (sizeof(SeqDesc) / 4) + (size_t)pages + n_items * (sizeof(AttnItem) / 4) + 64);
     l.meta = take(l.meta_bytes);
     l.total = at;
     return l;
@@ -164,6 +164,56 @@ int Forward::run_t(const CallDesc &call, float *scores, cudaStream_t stream, std
     const size_t o_score = call.score_off ? put(call.score_off, (size_t)B + 1) : 0;
     const size_t o_seq = put(reinterpret_cast<const int32_t *>(call.seqs.data()), (size_t)B * (sizeof(SeqDesc) / 4));
     const size_t o_pt = call.page_table.empty() ? 0 : put(call.page_table.data(), call.page_table.size());
+    // tensor-core attention work items (bf16 model): one per (user, head, 128-row tile[, KV split])
+    std::vector<AttnItem> items;
+    std::vector<AttnMerge> merges;
+    size_t o_items = 0, o_merges = 0;
+    if (sizeof(T) == 2) {
+        struct Tile { int seq, q0, n_q, nb; };
+        std::vector<Tile> tiles;
+        for (int u = 0; u < B; ++u) {
+            const SeqDesc &sd = call.seqs[(size_t)u];
+            const int nPB = (sd.n_paged + 127) / 128, nLB = (sd.n_lin + 127) / 128;
+            for (int q0 = 0; q0 < sd.n_q; q0 += 128) {
+                const int n_q = std::min(128, sd.n_q - q0);
+                const int tp1 = sd.q_pos0 + q0 + n_q - 1;
+                const int kmax = tp1 < sd.causal_end ? tp1 : sd.causal_end - 1;      // last key position any row of the tile sees
+                int nb = 0;
+                if (kmax >= 0) {
+                    const int pb = sd.n_paged > 0 ? std::min(nPB, kmax / 128 + 1) : 0;
+                    int lb = 0;
+                    if (pb == nPB && sd.n_lin > 0 && kmax >= sd.lin_pos0) lb = std::min(nLB, (kmax - sd.lin_pos0) / 128 + 1);
+                    nb = pb + lb;
+                }
+                tiles.push_back({u, q0, n_q, nb});
+            }
+        }
+        // split long key ranges when there are too few tiles to fill the GPU
+        const int64_t base = (int64_t)tiles.size() * H;
+        const int64_t target = 2 * (int64_t)n_sms;
+        int want = base > 0 && base < target ? (int)((target + base - 1) / base) : 1;
+        int part_slot = 0;
+        std::sort(tiles.begin(), tiles.end(), [](const Tile &x, const Tile &y) { return x.nb > y.nb; });   // longest first
+        for (const Tile &t : tiles) {
+            int ns = std::max(1, std::min(want, t.nb / 4));          // at least 4 key blocks per split
+            if (ns > 1 && part_slot + ns * H > kMaxSplitTiles) ns = 1;
+            const bool has_cand = call.seqs[(size_t)t.seq].q_pos0 + t.q0 + t.n_q > call.seqs[(size_t)t.seq].causal_end;
+            for (int h = 0; h < H; ++h) {
+                if (ns == 1) {
+                    items.push_back({t.seq, h, t.q0, t.n_q, 0, t.nb, -1, has_cand ? 1 : 0});
+                } else {
+                    merges.push_back({t.seq, h, t.q0, t.n_q, part_slot, ns});
+                    for (int i = 0; i < ns; ++i) {
+                        const int b0 = (int)((int64_t)t.nb * i / ns), b1 = (int)((int64_t)t.nb * (i + 1) / ns);
+                        items.push_back({t.seq, h, t.q0, t.n_q, b0, b1, part_slot + i, (i == 0 && has_cand) ? 1 : 0});
+                    }
+                    part_slot += ns;
+                }
+            }
+        }
+        if (!items.empty()) o_items = put(reinterpret_cast<const int32_t *>(items.data()), items.size() * (sizeof(AttnItem) / 4));
+        if (!merges.empty()) o_merges = put(reinterpret_cast<const int32_t *>(merges.data()), merges.size() * (sizeof(AttnMerge) / 4));
+    }
     if (blob.size() * 4 > lay.meta_bytes) { err = "internal: metadata larger than its workspace region"; return RELAYGR_E_NOSPACE; }
     int rc = upload(blob, lay.meta, stream, err);
     if (rc) return rc;
@@ -192,11 +242,18 @@ int Forward::run_t(const CallDesc &call, float *scores, cudaStream_t stream, std
     // bf16 model: GEMMs and attention run on the tensor cores; per-call tensor maps of the activations
     constexpr bool kTensor = sizeof(T) == 2;
     int *d_status = reinterpret_cast<int *>(ws + lay.status);
-    CUtensorMap tm_a, tm_att, tm_hid;
+    CUtensorMap tm_a, tm_att, tm_hid, tm_q, tm_k, tm_v, tm_pool;
     if (kTensor) {
         int trc = make_tmap_2d_bf16(&tm_a, a, (uint64_t)R, (uint64_t)d, (uint64_t)d, 128, 64);
         trc |= make_tmap_2d_bf16(&tm_att, att, (uint64_t)R, (uint64_t)d, (uint64_t)d, 128, 64);
         trc |= make_tmap_2d_bf16(&tm_hid, hid, (uint64_t)R, (uint64_t)F, (uint64_t)F, 128, 64);
+        trc |= make_tmap_2d_bf16(&tm_q, q, (uint64_t)R, (uint64_t)d, (uint64_t)d, 128, 64);
+        trc |= make_tmap_2d_bf16(&tm_k, kl, (uint64_t)R, (uint64_t)d, (uint64_t)d, 64, 64);
+        trc |= make_tmap_2d_bf16(&tm_v, vl, (uint64_t)R, (uint64_t)d, (uint64_t)d, 64, 64);
+        if (call.pool_slab)
+            trc |= make_tmap_2d_bf16(&tm_pool, call.pool_slab, (uint64_t)call.pool_pages * L * 2 * 64, (uint64_t)d, (uint64_t)d, 64, 64);
+        else
+            tm_pool = tm_k;
         if (trc != 0) { err = "tensor-map encoding of the activations failed"; return RELAYGR_E_CUDA; }
     }
     auto gemm = [&](const T *A, const CUtensorMap &tmA, const T *W, const CUtensorMap *tmW, int N, int K, const Epilogue &ep) {
@@ -231,7 +288,12 @@ int Forward::run_t(const CallDesc &call, float *scores, cudaStream_t stream, std
         if (!ck("QKV projection")) return RELAYGR_E_CUDA;
         if (kv_only) break;
 
-        e = launch_attention_simt<T>(q, kl, vl, paged, d_seqs, d_row_off, B, R, H, cfg.d_head, att, stream, &launches);
+        if constexpr (kTensor)
+            e = launch_attention_tc(tm_q, tm_k, tm_v, tm_pool, reinterpret_cast<const AttnItem *>(meta + o_items), (int)items.size(),
+                                    reinterpret_cast<const AttnMerge *>(meta + o_merges), (int)merges.size(), d_seqs, meta + o_pt, L, l,
+                                    d, q, kl, vl, att, reinterpret_cast<float *>(ws + lay.partial), d_status, stream, &launches);
+        else
+            e = launch_attention_simt<T>(q, kl, vl, paged, d_seqs, d_row_off, B, R, H, cfg.d_head, att, stream, &launches);
         if (!ck("attention")) return RELAYGR_E_CUDA;
 
         Epilogue eo{};

@@ -33,15 +33,6 @@ struct WorkspaceLayout {
     size_t meta_bytes, partial_bytes;
 };
 
-// One unit of tensor-core attention work: a 128-row query tile of one head of one
-// user against a contiguous range of that user's 128-key blocks.
-struct AttnWork {
-    int32_t seq, head, q0, n_q;          // query rows q0 .. q0+n_q-1 of the user (local index)
-    int32_t blk0, blk1;                  // key blocks [blk0, blk1) in the order: paged blocks, then linear blocks
-    int32_t partial_slot;                // >= 0: write (m, l, O) partials here instead of the output
-    int32_t n_splits;
-};
-
 struct Forward {
     relaygr_model_cfg cfg{};
     relaygr_weights w{};

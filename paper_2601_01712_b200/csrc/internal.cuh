@@ -37,6 +37,21 @@ struct PagedKV {
     int32_t n_layers, d_model, layer;
 };
 
+// One unit of tensor-core attention work: a 128-row query tile of one head of one user
+// against the key blocks [blk0, blk1) of that user (128 keys each; paged blocks first,
+// then linear blocks).  partial_slot >= 0: write (m, l, O) to that slot for a later merge.
+struct AttnItem {
+    int32_t seq, head, q0, n_q;
+    int32_t blk0, blk1;
+    int32_t partial_slot;
+    int32_t with_self;        // fold the candidate's own key in (exactly one split of a tile does)
+};
+
+struct AttnMerge {
+    int32_t seq, head, q0, n_q;
+    int32_t slot0, n_splits;
+};
+
 enum EpiMode : int32_t { EPI_STORE = 0, EPI_RESID = 1, EPI_QKV = 2 };
 
 // What a GEMM does with its fp32 accumulators: C[m, n] = sum_k A[m,k] W[n,k].

@@ -52,4 +52,13 @@ cudaError_t launch_attention_simt(const T *q, const T *k_lin, const T *v_lin, Pa
 cudaError_t launch_gemm_tc(const CUtensorMap &tmA, const CUtensorMap &tmB, int64_t M, int N, int K, const Epilogue &epi,
                            int *err, cudaStream_t stream, int64_t *launches);
 
+// Flash-style attention on tcgen05 (d_head = 64) over the work items, then the merge of split items.
+// tmQ: [rows, d] box 128 x 64; tmK / tmV: the call's transient K / V rows, box 64 x 64; tmPool: the pool
+// slab viewed as [pages * L * 2 * 64, d], box 64 x 64 (pass tmK when the call has no pool).
+cudaError_t launch_attention_tc(const CUtensorMap &tmQ, const CUtensorMap &tmK, const CUtensorMap &tmV, const CUtensorMap &tmPool,
+                                const AttnItem *items, int n_items, const AttnMerge *merges, int n_merges, const SeqDesc *seqs,
+                                const int32_t *pt, int n_layers, int layer, int d_model, const __nv_bfloat16 *q,
+                                const __nv_bfloat16 *k_lin, const __nv_bfloat16 *v_lin, __nv_bfloat16 *out, float *partial,
+                                int *err, cudaStream_t stream, int64_t *launches);
+
 }  // namespace relaygr
