@@ -1,0 +1,342 @@
+#!/usr/bin/env python
+"""Benchmark of the relay-race GR inference hot path on B200.
+
+One step = one ``relaygr_rank`` call over a batch of the production-shaped workload
+(32 users x 2048-token prefix already pre-inferred into the paged pool, 64 short-term
+tokens, 512 candidates per user).  The prefix pre-infer and the full recompute of the
+same batch are timed beside it and reported in the same JSON line.  Prints ONE JSON line.
+
+    python bench.py --gpus 1 --steps 500 --warmup 20
+    python -m torch.distributed.run --nproc-per-node N ... bench.py --gpus N ...   (N independent replicas)
+    python bench.py --impl reference      (the CPU checker timed on the host cores)
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "candidates ranked/s with cached prefix KV (rank on cache); p50/p99 rank latency vs full recompute"
+UNIT = "candidates/s"
+WORKLOAD = "config2: 4 layers, d_model 256, 4 heads x 64, FFN 1024, bf16; 32 users x (prefix 2048 cached, 64 short-term, 512 candidates); Zipf(1.1) ids over 1M items"
+
+# dram__bytes_read.sum + dram__bytes_write.sum of one attention launch of this workload (ncu; see profiles/)
+ATTENTION_DRAM_TRAFFIC_BYTES = None
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return {"hbm_gbs": p["hbm_gbs"], "tflops": p.get("bf16_tflops_sustained", p["bf16_tflops"]),
+                "tflops_burst": p["bf16_tflops"], "source": "measured (MEASURED_PEAKS.json, sustained bf16)"}
+    return {"hbm_gbs": 6650.0, "tflops": 1400.0, "tflops_burst": 1590.0, "source": "fallback (earlier pool measurement)"}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+            except Exception:
+                continue
+            for name, v in zip(["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"], r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def reference_arm(args):
+    """The CPU checker as it stands, timed on the host cores on a bounded sample of the same workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import ref
+    from paper_2601_01712_b200 import synth
+    wl = synth.workload(2)
+    shape = wl.model
+    vocab = 50_000       # the sample touches few distinct ids; a smaller table keeps host set-up short
+    w = synth.make_weights(shape, wl.seed, vocab=vocab)
+    om = ref.Model(shape.n_layers, shape.d_model, shape.n_heads, shape.d_head, shape.d_ff, shape.ln_eps, {**w.mat, **w.vec})
+    rng = np.random.default_rng(wl.seed)
+    zipf = synth.ZipfIds(vocab, wl.zipf_a)
+    P, S, C = 2048, 64, 512
+    K, V = om.preinfer(zipf.draw(rng, P))        # not timed: the prefix is cached
+    for _ in range(min(args.warmup, 1)):
+        om.rank_cached(K, V, zipf.draw(rng, S), zipf.draw(rng, C))
+    steps = max(1, min(args.steps, 3))
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        om.rank_cached(K, V, zipf.draw(rng, S), zipf.draw(rng, C))
+    dt = (time.perf_counter() - t0) / steps
+    val = C / dt
+    sample = "1 user per step (prefix 2048 cached by the checker's own pre-infer, 64 short-term, 512 candidates), %d steps" % steps
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
+        "warmup": min(args.warmup, 1), "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": {"workload": WORKLOAD, "sample": sample},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": ref.n_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=500)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="ours")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--users", type=int, default=32)
+    ap.add_argument("--prefix", type=int, default=2048)
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return reference_arm(args)
+    args.warmup = max(args.warmup, 3)
+
+    import torch
+    from paper_2601_01712_b200 import build as libbuild
+    libbuild.build()
+    from paper_2601_01712_b200 import binding as B
+    from paper_2601_01712_b200 import synth, workloads
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist_mod.init_process_group("nccl", device_id=torch.device("cuda", local))
+        dist = dist_mod
+
+    wl = synth.workload(2)
+    shape = wl.model
+    n_users, P, S, C = args.users, args.prefix, 64, 512
+    # replicas: every rank holds its own users (user-hash placement), no data-path collective
+    built = workloads.build(shape, wl.seed + 1000 * rank, [P] * n_users, [S] * n_users, [C] * n_users, n_rotations=8,
+                            first_user=rank * n_users, device="cuda:%d" % local)
+    model, pool = built.model, built.pool
+    stream = torch.cuda.current_stream()
+    n_cand = n_users * C
+    scores = torch.empty(n_cand, dtype=torch.float32, device=model.device)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(ms):
+        if dist is None:
+            return ms
+        t = torch.tensor([ms], dtype=torch.float64, device=model.device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    # ---- pre-infer (timed beside the metric) --------------------------------------------------------
+    pre_steps = max(3, min(20, args.steps // 20))
+    pool.preinfer(built.dev_batches[0])
+    for _ in range(3):
+        workloads.realloc_users(built)
+        pool.preinfer(built.dev_batches[0])
+    torch.cuda.synchronize()
+    pre_ms = []
+    for _ in range(pre_steps):
+        workloads.realloc_users(built)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        pool.preinfer(built.dev_batches[0])
+        e1.record(stream)
+        e1.synchronize()
+        pre_ms.append(e0.elapsed_time(e1))
+    pre_ms_med = float(np.median(pre_ms))
+
+    # ---- rank on cache: the metric ------------------------------------------------------------------
+    nrot = len(built.dev_batches)
+    for i in range(args.warmup):
+        pool.rank(built.dev_batches[i % nrot], scores)
+    launches0 = model.launch_count()
+    sampler = ClockSampler(local)
+    barrier()
+    sampler.start()
+    evs = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+    evs[0].record(stream)
+    for i in range(args.steps):
+        pool.rank(built.dev_batches[i % nrot], scores)
+        evs[i + 1].record(stream)
+    barrier()
+    clocks = sampler.stop()
+    total_ms = max_over_ranks(evs[0].elapsed_time(evs[-1]))
+    lat = np.array([evs[i].elapsed_time(evs[i + 1]) for i in range(args.steps)])
+    launches = model.launch_count() - launches0
+    assert model.device_status() == 0, "a kernel reported an internal error"
+    ms_per_step = total_ms / args.steps
+    value = world * n_cand / (ms_per_step * 1e-3)
+
+    # one call at a time (stream idle before each call): per-call latency as a request sees it
+    lat1 = []
+    for i in range(min(args.steps, 200)):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record(stream)
+        pool.rank(built.dev_batches[i % nrot], scores)
+        e1.record(stream)
+        e1.synchronize()
+        lat1.append(e0.elapsed_time(e1))
+    lat1 = np.array(lat1)
+
+    # ---- full recompute of the same batches ---------------------------------------------------------
+    full_steps = max(5, min(100, args.steps // 5))
+    for i in range(3):
+        model.rank_full(built.dev_batches[i % nrot], scores)
+    torch.cuda.synchronize()
+    full_lat = []
+    for i in range(full_steps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        model.rank_full(built.dev_batches[i % nrot], scores)
+        e1.record(stream)
+        e1.synchronize()
+        full_lat.append(e0.elapsed_time(e1))
+    full_lat = np.array(full_lat)
+
+    # ---- per-kernel timing of the rank step (events around every launch; separate from the timed region)
+    B.relaygr_profile_enable(model.ctx, True)
+    prof_steps = min(args.steps, 50)
+    for i in range(prof_steps):
+        pool.rank(built.dev_batches[i % nrot], scores)
+    prof = B.relaygr_profile_read(model.ctx)
+    B.relaygr_profile_enable(model.ctx, False)
+    attn_ms = prof["attention_ms"] / max(1, prof["attention_launches"])
+    attn_flops = workloads.attention_flops_per_layer(shape, built.batches[0], "rank")
+    peaks = load_peaks()
+    attn_tflops = attn_flops / (attn_ms * 1e-3) / 1e12
+    prof_total = sum(prof[k] for k in prof if k.endswith("_ms"))
+
+    # ---- end to end through host buffers ------------------------------------------------------------
+    hb = [(torch.from_numpy(b.short_ids).pin_memory(), torch.from_numpy(b.cand_ids).pin_memory()) for b in built.batches]
+    d_short = torch.empty_like(built.dev_batches[0].short_ids)
+    d_cand = torch.empty_like(built.dev_batches[0].cand_ids)
+    h_scores = torch.empty(n_cand, dtype=torch.float32).pin_memory()
+    b0 = built.batches[0]
+    ctx, kp = model.ctx, pool.pool
+
+    def e2e_step(i):
+        hs, hc = hb[i % nrot]
+        d_short.copy_(hs, non_blocking=True)
+        d_cand.copy_(hc, non_blocking=True)
+        B.relaygr_rank(ctx, kp, b0.users, d_short.data_ptr(), b0.short_off, d_cand.data_ptr(), b0.cand_off,
+                       scores.data_ptr(), stream.cuda_stream)
+        h_scores.copy_(scores, non_blocking=True)
+        stream.synchronize()
+
+    for i in range(5):
+        e2e_step(i)
+    e2e_steps = min(args.steps, 200)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for i in range(e2e_steps):
+        e2e_step(i)
+    e1.record(stream)
+    barrier()
+    e2e_ms = max_over_ranks(e0.elapsed_time(e1)) / e2e_steps
+    e2e = {"value": world * n_cand / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
+           "h2d_bytes_per_step": int(hb[0][0].numel() * 4 + hb[0][1].numel() * 4), "d2h_bytes_per_step": int(n_cand * 4)}
+
+    # ---- CPU baseline: the checker, timed on this machine's host cores ----------------------------------
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        from oracle import ref
+        om = ref.Model(shape.n_layers, shape.d_model, shape.n_heads, shape.d_head, shape.d_ff, shape.ln_eps,
+                       {**built.weights.mat, **built.weights.vec})
+        n_sample = 2
+        t_cpu, err = 0.0, 0.0
+        got = None
+        pool.rank(built.dev_batches[0], scores)
+        got = scores.cpu().numpy()
+        for u in range(n_sample):
+            p, s, c = b0.user_slices(u)
+            K, V = om.preinfer(p)
+            t0 = time.perf_counter()
+            want = om.rank_cached(K, V, s, c)
+            t_cpu += time.perf_counter() - t0
+            err = max(err, float(np.max(np.abs(got[b0.cand_off[u]:b0.cand_off[u + 1]] - want))))
+        cpu = {"value": n_sample * C / t_cpu, "unit": UNIT, "cores": ref.n_threads(), "kind": "oracle",
+               "sample": "%d of the %d users of one batch, rank on cache only (prefix K/V from the checker's own pre-infer, untimed)" % (n_sample, n_users),
+               "max_abs_err_vs_gpu": err}
+
+    if rank == 0:
+        rank_flops = workloads.batch_flops(shape, b0, "rank")
+        pre_flops = workloads.batch_flops(shape, b0, "preinfer")
+        full_flops = workloads.batch_flops(shape, b0, "full")
+        out = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "step": "one relaygr_rank call over the batch, prefix KV already in the paged pool",
+                       "users": n_users, "prefix": P, "short": S, "candidates": C,
+                       "l2": "inputs larger than L2: each step streams %.0f MiB of prefix K/V and rotates 8 input sets" % (n_users * shape.kv_bytes(P) / 2**20),
+                       "parallelism": "replicas (users hashed to GPUs), no collective" if world > 1 else "single GPU"},
+            "latency_ms": {"rank_p50_backlogged": float(np.percentile(lat, 50)), "rank_p99_backlogged": float(np.percentile(lat, 99)),
+                           "rank_p50": float(np.percentile(lat1, 50)), "rank_p99": float(np.percentile(lat1, 99)),
+                           "full_recompute_p50": float(np.percentile(full_lat, 50)), "full_recompute_p99": float(np.percentile(full_lat, 99)),
+                           "rank_beats_full_recompute_p99": bool(np.percentile(lat1, 99) < np.percentile(full_lat, 99))},
+            "preinfer": {"tokens_per_s": n_users * P / (pre_ms_med * 1e-3), "ms": pre_ms_med,
+                         "frac_of_tensor_roofline": pre_flops / (pre_ms_med * 1e-3) / 1e12 / peaks["tflops"]},
+            "whole_step_roofline": {"rank_tflops": rank_flops / (ms_per_step * 1e-3) / 1e12,
+                                    "rank_frac": rank_flops / (ms_per_step * 1e-3) / 1e12 / peaks["tflops"],
+                                    "full_recompute_tflops": full_flops / (float(np.median(full_lat)) * 1e-3) / 1e12},
+            "roofline": {"kernel": "attention_tc_kernel (rank)", "bound": "tensor", "achieved": attn_tflops, "peak": peaks["tflops"],
+                         "unit": "TFLOP/s", "frac": attn_tflops / peaks["tflops"], "peak_source": peaks["source"],
+                         "traffic": ATTENTION_DRAM_TRAFFIC_BYTES, "ms_per_launch": attn_ms,
+                         "algorithmic_flops_per_launch": attn_flops,
+                         "share_of_step": prof["attention_ms"] / prof_total if prof_total else None},
+            "kernel_ms_per_step": {k: prof[k] / prof_steps for k in prof if k.endswith("_ms")},
+            "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks, "cpu_baseline": cpu,
+        }
+        print(json.dumps(out))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -254,6 +254,21 @@ int32_t relaygr_rank_full(relaygr_ctx *ctx, int32_t n_users,
                           float *scores, void *stream);
 
 /*
+ * Per-kernel timing for benchmarks.  While enabled, every launch of a compute call is
+ * bracketed by CUDA events on the call's stream (a few microseconds of overhead per
+ * launch: do not leave it on for latency measurements).  relaygr_profile_read waits for
+ * the recorded events, returns device milliseconds and launch counts per kernel class
+ * accumulated since the previous read, and clears them.  "attention" covers the attention
+ * kernel and, when a call splits the key range, its merge kernel.
+ */
+typedef struct {
+    double gather_ln_ms, layernorm_ms, gemm_ms, attention_ms, score_ms;
+    int64_t gather_ln_launches, layernorm_launches, gemm_launches, attention_launches, score_launches;
+} relaygr_profile;
+int32_t relaygr_profile_enable(relaygr_ctx *ctx, int32_t on);
+int32_t relaygr_profile_read(relaygr_ctx *ctx, relaygr_profile *out);
+
+/*
  * Kernel launches enqueued by this ctx so far (for benchmark bookkeeping).
  */
 int32_t relaygr_launch_count(const relaygr_ctx *ctx, int64_t *out);

@@ -44,6 +44,15 @@ class PoolStats(C.Structure):
         return {n: int(getattr(self, n)) for n, _ in self._fields_}
 
 
+class Profile(C.Structure):
+    _fields_ = [(n, C.c_double) for n in ["gather_ln_ms", "layernorm_ms", "gemm_ms", "attention_ms", "score_ms"]] + \
+               [(n, C.c_int64) for n in ["gather_ln_launches", "layernorm_launches", "gemm_launches",
+                                         "attention_launches", "score_launches"]]
+
+    def as_dict(self):
+        return {n: getattr(self, n) for n, _ in self._fields_}
+
+
 class RelayGRError(RuntimeError):
     def __init__(self, code, msg):
         super().__init__("%s: %s" % (STATUS_NAMES.get(code, code), msg))
@@ -76,6 +85,8 @@ SIGNATURES = {
     "relaygr_preinfer": (_I32, [_P, _P, _I32, _P, _P, _P, _P]),
     "relaygr_rank": (_I32, [_P, _P, _I32, _P, _P, _P, _P, _P, _P, _P, _P]),
     "relaygr_rank_full": (_I32, [_P, _I32, _P, _P, _P, _P, _P, _P, _P, _P]),
+    "relaygr_profile_enable": (_I32, [_P, _I32]),
+    "relaygr_profile_read": (_I32, [_P, C.POINTER(Profile)]),
     "relaygr_launch_count": (_I32, [_P, C.POINTER(_I64)]),
 }
 
@@ -246,6 +257,16 @@ def relaygr_rank_full(ctx, n_users, prefix_ids_dev, prefix_off, short_ids_dev, s
     po, so, co = _host_i32(prefix_off), _host_i32(short_off), _host_i32(cand_off)
     return _check(lib().relaygr_rank_full(ctx, n_users, _ptr(prefix_ids_dev), _ptr(po), _ptr(short_ids_dev), _ptr(so),
                                           _ptr(cand_ids_dev), _ptr(co), _ptr(scores_dev), stream), ok)
+
+
+def relaygr_profile_enable(ctx, on: bool):
+    _check(lib().relaygr_profile_enable(ctx, int(on)))
+
+
+def relaygr_profile_read(ctx) -> dict:
+    out = Profile()
+    _check(lib().relaygr_profile_read(ctx, C.byref(out)))
+    return out.as_dict()
 
 
 def relaygr_launch_count(ctx) -> int:

@@ -13,8 +13,47 @@ inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 std::string cuda_msg(const char *what, cudaError_t e) { return std::string(what) + ": " + cudaGetErrorString(e); }
 }  // namespace
 
+cudaEvent_t Forward::prof_begin(cudaStream_t stream)
+{
+    if (!profiling) return nullptr;
+    cudaEvent_t ev = nullptr;
+    if (!prof_spare.empty()) { ev = prof_spare.back(); prof_spare.pop_back(); }
+    else if (cudaEventCreate(&ev) != cudaSuccess) return nullptr;
+    cudaEventRecord(ev, stream);
+    return ev;
+}
+
+void Forward::prof_end(int cls, cudaEvent_t start, cudaStream_t stream)
+{
+    if (!start) return;
+    cudaEvent_t ev = nullptr;
+    if (!prof_spare.empty()) { ev = prof_spare.back(); prof_spare.pop_back(); }
+    else if (cudaEventCreate(&ev) != cudaSuccess) { prof_spare.push_back(start); return; }
+    cudaEventRecord(ev, stream);
+    prof_pending[cls].push_back({start, ev});
+}
+
+int Forward::profile_read(double *ms, int64_t *count, std::string &err)
+{
+    for (int c = 0; c < KC_COUNT; ++c) {
+        ms[c] = 0.0; count[c] = 0;
+        for (const EvPair &p : prof_pending[c]) {
+            cudaError_t e = cudaEventSynchronize(p.b);
+            float t = 0.f;
+            if (e == cudaSuccess) e = cudaEventElapsedTime(&t, p.a, p.b);
+            if (e != cudaSuccess) { err = cuda_msg("profile read", e); return RELAYGR_E_CUDA; }
+            ms[c] += t; count[c] += 1;
+            prof_spare.push_back(p.a); prof_spare.push_back(p.b);
+        }
+        prof_pending[c].clear();
+    }
+    return RELAYGR_OK;
+}
+
 Forward::~Forward()
 {
+    for (int c = 0; c < KC_COUNT; ++c) for (const EvPair &p : prof_pending[c]) { cudaEventDestroy(p.a); cudaEventDestroy(p.b); }
+    for (cudaEvent_t ev : prof_spare) cudaEventDestroy(ev);
     for (int i = 0; i < kSlots; ++i) if (slot_event[i]) cudaEventDestroy(slot_event[i]);
     if (staging) cudaFreeHost(staging);
 }
@@ -257,15 +296,30 @@ int Forward::run_t(const CallDesc &call, float *scores, cudaStream_t stream, std
         if (trc != 0) { err = "tensor-map encoding of the activations failed"; return RELAYGR_E_CUDA; }
     }
     auto gemm = [&](const T *A, const CUtensorMap &tmA, const T *W, const CUtensorMap *tmW, int N, int K, const Epilogue &ep) {
-        if constexpr (kTensor) return launch_gemm_tc(tmA, *tmW, R, N, K, ep, d_status, stream, &launches);
-        else return launch_gemm_simt<T>(A, W, R, N, K, ep, stream, &launches);
+        cudaEvent_t pe = prof_begin(stream);
+        cudaError_t r;
+        if constexpr (kTensor) r = launch_gemm_tc(tmA, *tmW, R, N, K, ep, d_status, stream, &launches);
+        else r = launch_gemm_simt<T>(A, W, R, N, K, ep, stream, &launches);
+        prof_end(KC_GEMM, pe, stream);
+        return r;
+    };
+    auto layernorm = [&](const float *g, const float *b) {
+        cudaEvent_t pe = prof_begin(stream);
+        const cudaError_t r = launch_layernorm<T>(x, d, R, g, b, cfg.ln_eps, a, stream, &launches);
+        prof_end(KC_LAYERNORM, pe, stream);
+        return r;
     };
     const LayerMaps *lm = nullptr;
 
     for (int l = 0; l < L; ++l) {
         const float *g1 = w.ln1_g + (size_t)l * d, *b1n = w.ln1_b + (size_t)l * d;
-        if (l == 0) e = launch_gather_ln<T>((const T *)w.emb, cfg.vocab, d, src, R, g1, b1n, cfg.ln_eps, x, a, stream, &launches);
-        else e = launch_layernorm<T>(x, d, R, g1, b1n, cfg.ln_eps, a, stream, &launches);
+        if (l == 0) {
+            cudaEvent_t pe = prof_begin(stream);
+            e = launch_gather_ln<T>((const T *)w.emb, cfg.vocab, d, src, R, g1, b1n, cfg.ln_eps, x, a, stream, &launches);
+            prof_end(KC_GATHER_LN, pe, stream);
+        } else {
+            e = layernorm(g1, b1n);
+        }
         if (!ck("LayerNorm 1")) return RELAYGR_E_CUDA;
 
         // fused QKV projection; the last pre-infer layer only needs K and V (psi is K/V alone)
@@ -288,12 +342,16 @@ int Forward::run_t(const CallDesc &call, float *scores, cudaStream_t stream, std
         if (!ck("QKV projection")) return RELAYGR_E_CUDA;
         if (kv_only) break;
 
-        if constexpr (kTensor)
-            e = launch_attention_tc(tm_q, tm_k, tm_v, tm_pool, reinterpret_cast<const AttnItem *>(meta + o_items), (int)items.size(),
-                                    reinterpret_cast<const AttnMerge *>(meta + o_merges), (int)merges.size(), d_seqs, meta + o_pt, L, l,
-                                    d, q, kl, vl, att, reinterpret_cast<float *>(ws + lay.partial), d_status, stream, &launches);
-        else
-            e = launch_attention_simt<T>(q, kl, vl, paged, d_seqs, d_row_off, B, R, H, cfg.d_head, att, stream, &launches);
+        {
+            cudaEvent_t pe = prof_begin(stream);
+            if constexpr (kTensor)
+                e = launch_attention_tc(tm_q, tm_k, tm_v, tm_pool, reinterpret_cast<const AttnItem *>(meta + o_items), (int)items.size(),
+                                        reinterpret_cast<const AttnMerge *>(meta + o_merges), (int)merges.size(), d_seqs, meta + o_pt, L,
+                                        l, d, q, kl, vl, att, reinterpret_cast<float *>(ws + lay.partial), d_status, stream, &launches);
+            else
+                e = launch_attention_simt<T>(q, kl, vl, paged, d_seqs, d_row_off, B, R, H, cfg.d_head, att, stream, &launches);
+            prof_end(KC_ATTENTION, pe, stream);
+        }
         if (!ck("attention")) return RELAYGR_E_CUDA;
 
         Epilogue eo{};
@@ -301,7 +359,7 @@ int Forward::run_t(const CallDesc &call, float *scores, cudaStream_t stream, std
         e = gemm(att, tm_att, (const T *)w.w_o + (size_t)l * d * d, lm ? &lm->wo : nullptr, d, d, eo);
         if (!ck("output projection")) return RELAYGR_E_CUDA;
 
-        e = launch_layernorm<T>(x, d, R, w.ln2_g + (size_t)l * d, w.ln2_b + (size_t)l * d, cfg.ln_eps, a, stream, &launches);
+        e = layernorm(w.ln2_g + (size_t)l * d, w.ln2_b + (size_t)l * d);
         if (!ck("LayerNorm 2")) return RELAYGR_E_CUDA;
 
         Epilogue e1{};
@@ -316,8 +374,10 @@ int Forward::run_t(const CallDesc &call, float *scores, cudaStream_t stream, std
     }
 
     if (!preinfer && call.score_off && call.score_off[B] > 0) {
+        cudaEvent_t pe = prof_begin(stream);
         e = launch_score(x, d, d_seqs, B, call.score_off[B], meta + o_score, w.lnf_g, w.lnf_b, cfg.ln_eps, w.w_score, w.b_score,
                          scores, stream, &launches);
+        prof_end(KC_SCORE, pe, stream);
         if (!ck("scoring head")) return RELAYGR_E_CUDA;
     }
     return RELAYGR_OK;

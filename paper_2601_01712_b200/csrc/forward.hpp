@@ -54,6 +54,16 @@ struct Forward {
     bool slot_used[kSlots] = {};
     int next_slot = 0;
 
+    // optional per-kernel-class timing with CUDA events on the call's stream
+    enum KernelClass { KC_GATHER_LN = 0, KC_LAYERNORM, KC_GEMM, KC_ATTENTION, KC_SCORE, KC_COUNT };
+    bool profiling = false;
+    struct EvPair { cudaEvent_t a, b; };
+    std::vector<EvPair> prof_pending[KC_COUNT];
+    std::vector<cudaEvent_t> prof_spare;
+    cudaEvent_t prof_begin(cudaStream_t stream);
+    void prof_end(int cls, cudaEvent_t start, cudaStream_t stream);
+    int profile_read(double *ms, int64_t *count, std::string &err);
+
     ~Forward();
     int init_device(int dev, std::string &err);
     WorkspaceLayout layout(int64_t rows, int64_t users, int64_t pages) const;

@@ -137,6 +137,29 @@ int32_t relaygr_device_status(relaygr_ctx *ctx, void *stream, int32_t *out)
     return ctx->fwd.device_status((cudaStream_t)stream, out, g_err);
 }
 
+int32_t relaygr_profile_enable(relaygr_ctx *ctx, int32_t on)
+{
+    if (!ctx) return fail(RELAYGR_E_INVALID, "ctx is NULL");
+    ctx->fwd.profiling = on != 0;
+    return RELAYGR_OK;
+}
+
+int32_t relaygr_profile_read(relaygr_ctx *ctx, relaygr_profile *out)
+{
+    if (!ctx || !out) return fail(RELAYGR_E_INVALID, "bad argument");
+    std::memset(out, 0, sizeof(*out));
+    if (ctx->host_only) return RELAYGR_OK;
+    double ms[Forward::KC_COUNT]; int64_t n[Forward::KC_COUNT];
+    const int rc = ctx->fwd.profile_read(ms, n, g_err);
+    if (rc) return rc;
+    out->gather_ln_ms = ms[Forward::KC_GATHER_LN]; out->gather_ln_launches = n[Forward::KC_GATHER_LN];
+    out->layernorm_ms = ms[Forward::KC_LAYERNORM]; out->layernorm_launches = n[Forward::KC_LAYERNORM];
+    out->gemm_ms = ms[Forward::KC_GEMM]; out->gemm_launches = n[Forward::KC_GEMM];
+    out->attention_ms = ms[Forward::KC_ATTENTION]; out->attention_launches = n[Forward::KC_ATTENTION];
+    out->score_ms = ms[Forward::KC_SCORE]; out->score_launches = n[Forward::KC_SCORE];
+    return RELAYGR_OK;
+}
+
 int32_t relaygr_launch_count(const relaygr_ctx *ctx, int64_t *out)
 {
     if (!ctx || !out) return fail(RELAYGR_E_INVALID, "bad argument");
