@@ -26,8 +26,11 @@ def _deps_mtime() -> float:
 
 
 def build(force: bool = False, verbose: bool = False) -> str:
-    os.makedirs(OBJ, exist_ok=True)
     hdr_time = _deps_mtime()
+    newest = max([hdr_time] + [os.path.getmtime(s) for s in sources()])
+    if not force and os.path.exists(LIB) and os.path.getmtime(LIB) >= newest:
+        return LIB                      # up to date (object files are not needed to know that)
+    os.makedirs(OBJ, exist_ok=True)
     jobs = []
     objs = []
     for src in sources():
@@ -36,6 +39,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
         stale = force or not os.path.exists(obj) or os.path.getmtime(obj) < max(os.path.getmtime(src), hdr_time)
         if stale:
             extra = ["-Xptxas", "-v"] if verbose else []
+            extra += os.environ.get("RELAYGR_NVCC_EXTRA", "").split()
             jobs.append(["nvcc", *NVCC_FLAGS, *extra, "-x", "cu", "-c", src, "-o", obj])
 
     def run(cmd):

@@ -3,17 +3,21 @@
 // table + short-term rows + the candidate's own row) and full inference (linear K/V rows).
 //
 // One CTA = one work item: a 128-row query tile of one head of one user against a range of
-// that user's 128-key blocks.  Per block:  S = Q K^T  (tcgen05.mma, M=128 N=128 K=64, operands in
-// shared memory, S in TMEM) -> online softmax by 128 threads, one row each, P written back to
-// TMEM as bf16 -> O += P V (tcgen05.mma, M=128 N=64 K=128, A = P from TMEM, B = V in shared
-// memory, MN-major, O accumulated in TMEM).  The running maximum is only raised (and O rescaled
-// in TMEM) when it grows by more than 2^8, which keeps every exponent in range and makes the
-// rescale rare.  K/V tiles are two 64-row TMA boxes each: 64-token pages of the pool addressed
-// through the page table, or rows of the call's transient K/V buffers.
+// that user's 64-key blocks (one block = one 64-token page of the pool, or 64 rows of the
+// call's transient K/V buffers; one 8 KB TMA box each for K and V).  Per block:
+//     S = Q K^T   tcgen05.mma M=128 N=64 K=64, operands in shared memory, S in TMEM
+//     softmax     128 threads, one row each: S row -> registers, running max, p = 2^(s c - m c),
+//                 bf16 P written back to TMEM
+//     O += P V    tcgen05.mma M=128 N=64 K=64, A = P from TMEM, B = V in shared memory (MN-major),
+//                 O accumulated in TMEM
+// S and P are double-buffered in TMEM, so the MMA warp runs one block ahead of the softmax and
+// the tensor pipe never waits for it in steady state.  The running maximum is only raised (and
+// O rescaled in TMEM, after the pending PV has drained) when it grows by more than 2^8, which
+// keeps every exponent in range and makes the rescale rare.
 //
 // Warp roles (192 threads): warp 0 = TMA producer, warp 1 = TMEM owner + MMA issuer,
 // warps 2-5 = softmax / correction / epilogue (TMEM lane quadrant = warp index % 4).
-// Two CTAs per SM: one CTA's softmax overlaps the other's MMAs.
+// Two CTAs per SM.
 #include "kernels.cuh"
 #include "tc_common.cuh"
 
@@ -21,19 +25,19 @@ namespace relaygr {
 
 namespace {
 
-constexpr int kQTile = 128, kKeys = 128, kDh = 64;
+constexpr int kQTile = 128, kKeys = 64, kDh = 64;
 constexpr int kQBytes = kQTile * kDh * 2;           // 16 KB
-constexpr int kKVBytes = kKeys * kDh * 2;           // 16 KB per K or V tile (two 8 KB boxes)
-constexpr int kStagesKV = 2;
-constexpr int kSmemBytes = kQBytes + 2 * kStagesKV * kKVBytes + 1024 + 256;
-constexpr uint32_t kTmemCols = 256;                 // S: 0..127, P: 128..191, O: 192..255
+constexpr int kKVBytes = kKeys * kDh * 2;           // 8 KB per K or V tile
+constexpr int kStagesKV = 4;
+constexpr int kSmemBytes = kQBytes + 2 * kStagesKV * kKVBytes + 1024 + 512;
+constexpr uint32_t kTmemCols = 256;                 // S[2]: 0..127, P[2]: 128..191, O: 192..255
 constexpr uint32_t kColS = 0, kColP = 128, kColO = 192;
 constexpr float kRescaleThreshold = 8.f;            // in log2 units
 
 struct Bars {
     uint64_t q_full;
     uint64_t k_full[kStagesKV], k_empty[kStagesKV], v_full[kStagesKV], v_empty[kStagesKV];
-    uint64_t s_full, s_free, p_full, pv_done;
+    uint64_t s_full[2], s_free[2], p_full[2], p_free[2];
     uint32_t tmem_slot;
     int abort_flag;
 };
@@ -43,6 +47,12 @@ __device__ __forceinline__ float ex2(float x)
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
+}
+__device__ __forceinline__ float max3(float a, float b, float c)
+{
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
 }
 
 __global__ void __launch_bounds__(192, 2)
@@ -63,7 +73,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     const AttnItem it = items[blockIdx.x];
     const SeqDesc sd = seqs[it.seq];
     const int nb = it.blk1 - it.blk0;
-    const int n_paged_blocks = (sd.n_paged + kKeys - 1) / kKeys;
+    const int n_paged_blocks = (sd.n_paged + kKeys - 1) / kKeys;      // = the user's page count
 
     if (threadIdx.x == 0) bars->abort_flag = *reinterpret_cast<volatile int *>(err);
     __syncthreads();
@@ -75,10 +85,10 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             tc::mbar_init(&bars->k_full[s], 1); tc::mbar_init(&bars->k_empty[s], 1);
             tc::mbar_init(&bars->v_full[s], 1); tc::mbar_init(&bars->v_empty[s], 1);
         }
-        tc::mbar_init(&bars->s_full, 1);
-        tc::mbar_init(&bars->s_free, 128);
-        tc::mbar_init(&bars->p_full, 128);
-        tc::mbar_init(&bars->pv_done, 1);
+        for (int b = 0; b < 2; ++b) {
+            tc::mbar_init(&bars->s_full[b], 1); tc::mbar_init(&bars->s_free[b], 128);
+            tc::mbar_init(&bars->p_full[b], 128); tc::mbar_init(&bars->p_free[b], 1);
+        }
         tc::fence_mbar_init();
         tc::tma_prefetch_desc(&tmQ); tc::tma_prefetch_desc(&tmKlin); tc::tma_prefetch_desc(&tmVlin); tc::tma_prefetch_desc(&tmPool);
     }
@@ -100,64 +110,58 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 const int b = it.blk0 + j;
                 const int s = j % kStagesKV;
                 const uint32_t par = ((j / kStagesKV) & 1) ^ 1;
-                const bool paged = b < n_paged_blocks;
-                int y0, y1;              // first rows of the two 64-key halves (K); V rows follow from them
-                int vy0, vy1;
+                int ky, vy;
                 const CUtensorMap *mk, *mv;
-                if (paged) {
-                    const int p0 = pt[sd.pt_base + 2 * b];
-                    const bool two = (2 * b + 1) * 64 < sd.n_paged;
-                    const int p1 = two ? pt[sd.pt_base + 2 * b + 1] : p0;      // absent half: re-read the first page (masked later)
-                    y0 = ((p0 * n_layers + layer) * 2) * 64; y1 = ((p1 * n_layers + layer) * 2) * 64;
-                    vy0 = y0 + 64; vy1 = y1 + 64;
+                if (b < n_paged_blocks) {
+                    const int page = pt[sd.pt_base + b];
+                    ky = ((page * n_layers + layer) * 2) * 64; vy = ky + 64;
                     mk = &tmPool; mv = &tmPool;
                 } else {
-                    const int r = sd.lin_row0 + (b - n_paged_blocks) * kKeys;
-                    y0 = r; y1 = r + 64; vy0 = y0; vy1 = y1;
+                    ky = vy = sd.lin_row0 + (b - n_paged_blocks) * kKeys;
                     mk = &tmKlin; mv = &tmVlin;
                 }
                 if (!tc::mbar_wait(&bars->k_empty[s], par, err)) break;
                 tc::mbar_expect_tx(&bars->k_full[s], kKVBytes);
-                tc::tma_load_2d(sK + s * kKVBytes, mk, it.head * kDh, y0, &bars->k_full[s]);
-                tc::tma_load_2d(sK + s * kKVBytes + kKVBytes / 2, mk, it.head * kDh, y1, &bars->k_full[s]);
+                tc::tma_load_2d(sK + s * kKVBytes, mk, it.head * kDh, ky, &bars->k_full[s]);
                 if (!tc::mbar_wait(&bars->v_empty[s], par, err)) break;
                 tc::mbar_expect_tx(&bars->v_full[s], kKVBytes);
-                tc::tma_load_2d(sV + s * kKVBytes, mv, it.head * kDh, vy0, &bars->v_full[s]);
-                tc::tma_load_2d(sV + s * kKVBytes + kKVBytes / 2, mv, it.head * kDh, vy1, &bars->v_full[s]);
+                tc::tma_load_2d(sV + s * kKVBytes, mv, it.head * kDh, vy, &bars->v_full[s]);
             }
         }
     } else if (warp == 1) {
         // ---------------------------------------------------------------- MMA issuer
         if (lane == 0) {
-            constexpr uint32_t idesc_qk = tc::make_idesc(128, 128, 0, 0);     // Q, K both K-major
-            constexpr uint32_t idesc_pv = tc::make_idesc(128, 64, 0, 1);      // P from TMEM, V MN-major
+            constexpr uint32_t idesc_qk = tc::make_idesc(128, kKeys, 0, 0);   // Q, K both K-major
+            constexpr uint32_t idesc_pv = tc::make_idesc(128, kDh, 0, 1);     // P from TMEM, V MN-major
             const uint64_t qdesc = tc::smem_desc_sw128(tc::smem_u32(sQ));
             bool ok = tc::mbar_wait(&bars->q_full, 0, err);
-            auto issue_qk = [&](int j) {
-                const int s = j % kStagesKV;
+            auto issue_qk = [&](int j) {        // S[j & 1] = Q K(j)^T
+                const int s = j % kStagesKV, b = j & 1;
                 if (!tc::mbar_wait(&bars->k_full[s], (j / kStagesKV) & 1, err)) return false;
-                if (j > 0 && !tc::mbar_wait(&bars->s_free, (j - 1) & 1, err)) return false;
+                if (j >= 2 && !tc::mbar_wait(&bars->s_free[b], ((j >> 1) - 1) & 1, err)) return false;
                 tc::tc_fence_after();
                 const uint64_t kdesc = tc::smem_desc_sw128(tc::smem_u32(sK + s * kKVBytes));
 #pragma unroll
-                for (int k = 0; k < kDh / 16; ++k) tc::mma_ss(tmem_base + kColS, qdesc + 2 * k, kdesc + 2 * k, idesc_qk, k != 0);
-                tc::mma_commit(&bars->s_full);
+                for (int k = 0; k < kDh / 16; ++k)
+                    tc::mma_ss(tmem_base + kColS + b * kKeys, qdesc + 2 * k, kdesc + 2 * k, idesc_qk, k != 0);
+                tc::mma_commit(&bars->s_full[b]);
                 tc::mma_commit(&bars->k_empty[s]);
                 return true;
             };
             if (ok && nb > 0) ok = issue_qk(0);
+            if (ok && nb > 1) ok = issue_qk(1);
             for (int j = 0; j < nb && ok; ++j) {
-                if (j + 1 < nb) { ok = issue_qk(j + 1); if (!ok) break; }
-                const int s = j % kStagesKV;
-                if (!tc::mbar_wait(&bars->p_full, j & 1, err)) break;
+                const int s = j % kStagesKV, b = j & 1;
+                if (!tc::mbar_wait(&bars->p_full[b], (j >> 1) & 1, err)) break;
                 if (!tc::mbar_wait(&bars->v_full[s], (j / kStagesKV) & 1, err)) break;
                 tc::tc_fence_after();
                 const uint64_t vdesc = tc::smem_desc_sw128(tc::smem_u32(sV + s * kKVBytes));
 #pragma unroll
                 for (int k = 0; k < kKeys / 16; ++k)      // 16 keys per instruction: 8 TMEM columns of P, 2048 bytes of V
-                    tc::mma_ts(tmem_base + kColO, tmem_base + kColP + 8 * k, vdesc + 128 * k, idesc_pv, (j | k) != 0);
-                tc::mma_commit(&bars->pv_done);
+                    tc::mma_ts(tmem_base + kColO, tmem_base + kColP + b * (kKeys / 2) + 8 * k, vdesc + 128 * k, idesc_pv, (j | k) != 0);
+                tc::mma_commit(&bars->p_free[b]);          // P[b] consumed; also "O holds blocks 0..j"
                 tc::mma_commit(&bars->v_empty[s]);
+                if (j + 2 < nb) ok = issue_qk(j + 2);      // S[b] was freed by the softmax of block j
             }
         }
     } else {
@@ -174,91 +178,92 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         bool ok = true;
 
         for (int j = 0; j < nb && ok; ++j) {
-            const int b = it.blk0 + j;
-            const bool paged = b < n_paged_blocks;
-            const int kidx0 = paged ? b * kKeys : (b - n_paged_blocks) * kKeys;        // index of the block's first key in its source
+            const int blk = it.blk0 + j, b = j & 1;
+            const bool paged = blk < n_paged_blocks;
+            const int kidx0 = paged ? blk * kKeys : (blk - n_paged_blocks) * kKeys;    // index of the block's first key in its source
             const int kpos0 = paged ? kidx0 : sd.lin_pos0 + kidx0;                     // its sequence position
             const int n_valid = min(kKeys, (paged ? sd.n_paged : sd.n_lin) - kidx0);
             const bool need_mask = (n_valid < kKeys) || (kpos0 + kKeys - 1 > tile_min_lim);
             const int jmax = min(n_valid, lim - kpos0 + 1);  // keys jj < jmax of this block are visible to this row
 
-            ok = __all_sync(0xffffffffu, tc::mbar_wait(&bars->s_full, j & 1, err));
+            ok = __all_sync(0xffffffffu, tc::mbar_wait(&bars->s_full[b], (j >> 1) & 1, err));
             if (!ok) break;
             tc::tc_fence_after();
 
-            // pass 1: row maximum
-            float mx = -INFINITY;
-#pragma unroll 1
-            for (int cc = 0; cc < kKeys; cc += 32) {
-                uint32_t sv[32];
-                tc::tmem_ld32(lane_addr + kColS + cc, sv);
-                tc::tmem_ld_wait();
-                if (need_mask) {
+            // the S row of this block, in registers
+            uint32_t s0[32], s1[32];
+            tc::tmem_ld32(lane_addr + kColS + b * kKeys, s0);
+            tc::tmem_ld32(lane_addr + kColS + b * kKeys + 32, s1);
+            tc::tmem_ld_wait();
+            tc::tc_fence_before();
+            tc::mbar_arrive(&bars->s_free[b]);               // S[b] may be overwritten by the QK^T of block j + 2
+            if (need_mask) {
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) mx = fmaxf(mx, (cc + i < jmax) ? __uint_as_float(sv[i]) : -INFINITY);
-                } else {
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(sv[i]));
+                for (int i = 0; i < 32; ++i) {
+                    if (i >= jmax) s0[i] = 0xff800000u;      // -inf
+                    if (32 + i >= jmax) s1[i] = 0xff800000u;
                 }
+            }
+            float mx = -INFINITY;
+#pragma unroll
+            for (int i = 0; i < 32; i += 2) {
+                mx = max3(mx, __uint_as_float(s0[i]), __uint_as_float(s0[i + 1]));
+                mx = max3(mx, __uint_as_float(s1[i]), __uint_as_float(s1[i + 1]));
             }
             // raise the running maximum only when it grows by more than the threshold
             float alpha = 1.f;
-            bool raise = (mx - m) * c > kRescaleThreshold;          // false when mx == -inf; true on the first visible key
+            const bool raise = (mx - m) * c > kRescaleThreshold;    // false when mx == -inf; true on the first visible key
             if (raise) {
                 alpha = (m == -INFINITY) ? 0.f : ex2((m - mx) * c);
                 m = mx;
             }
             const float mc = (m == -INFINITY) ? 0.f : m * c;
-
-            // P(j) overwrites P(j-1) and the correction touches O: both need PV(j-1) complete
-            if (j > 0) {
-                ok = __all_sync(0xffffffffu, tc::mbar_wait(&bars->pv_done, (j - 1) & 1, err));
+            if (j > 0 && __any_sync(0xffffffffu, raise)) {
+                // correction: O must hold blocks 0..j-1 completely before it is rescaled
+                ok = __all_sync(0xffffffffu, tc::mbar_wait(&bars->p_free[(j - 1) & 1], ((j - 1) >> 1) & 1, err));
                 if (!ok) break;
                 tc::tc_fence_after();
-                if (__any_sync(0xffffffffu, raise)) {
 #pragma unroll 1
-                    for (int cc = 0; cc < kDh; cc += 16) {
-                        uint32_t ov[16];
-                        tc::tmem_ld16(lane_addr + kColO + cc, ov);
-                        tc::tmem_ld_wait();
+                for (int cc = 0; cc < kDh; cc += 16) {
+                    uint32_t ov[16];
+                    tc::tmem_ld16(lane_addr + kColO + cc, ov);
+                    tc::tmem_ld_wait();
 #pragma unroll
-                        for (int i = 0; i < 16; ++i) ov[i] = __float_as_uint(__uint_as_float(ov[i]) * alpha);
-                        tc::tmem_st16(lane_addr + kColO + cc, ov);
-                    }
+                    for (int i = 0; i < 16; ++i) ov[i] = __float_as_uint(__uint_as_float(ov[i]) * alpha);
+                    tc::tmem_st16(lane_addr + kColO + cc, ov);
                 }
             }
             l *= alpha;
-
-            // pass 2: p = 2^(s c - m c), row sum, bf16 P into TMEM
-            float rs = 0.f;
-#pragma unroll 1
-            for (int cc = 0; cc < kKeys; cc += 32) {
-                uint32_t sv[32];
-                tc::tmem_ld32(lane_addr + kColS + cc, sv);
-                tc::tmem_ld_wait();
-                float p[32];
-                if (need_mask) {
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) p[i] = (cc + i < jmax) ? ex2(fmaf(__uint_as_float(sv[i]), c, -mc)) : 0.f;
-                } else {
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) p[i] = ex2(fmaf(__uint_as_float(sv[i]), c, -mc));
-                }
-                uint32_t pk[16];
-#pragma unroll
-                for (int i = 0; i < 16; ++i) { rs += p[2 * i] + p[2 * i + 1]; pk[i] = tc::pack_bf16(p[2 * i], p[2 * i + 1]); }
-                tc::tmem_st16(lane_addr + kColP + cc / 2, pk);
+            // P[b] was last read by the PV of block j - 2
+            if (j >= 2) {
+                ok = __all_sync(0xffffffffu, tc::mbar_wait(&bars->p_free[b], ((j >> 1) - 1) & 1, err));
+                if (!ok) break;
             }
-            l += rs;
-            tc::tc_fence_before();
-            tc::mbar_arrive(&bars->s_free);        // S(j) fully read: the next QK^T may overwrite it
+            // p = 2^(s c - m c); row sum in fp32; bf16 P into TMEM
+            float rs0 = 0.f, rs1 = 0.f;
+            uint32_t pk[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                const float p0 = ex2(fmaf(__uint_as_float(s0[2 * i]), c, -mc)), p1 = ex2(fmaf(__uint_as_float(s0[2 * i + 1]), c, -mc));
+                rs0 += p0; rs1 += p1;
+                pk[i] = tc::pack_bf16(p0, p1);
+            }
+            tc::tmem_st16(lane_addr + kColP + b * (kKeys / 2), pk);
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                const float p0 = ex2(fmaf(__uint_as_float(s1[2 * i]), c, -mc)), p1 = ex2(fmaf(__uint_as_float(s1[2 * i + 1]), c, -mc));
+                rs0 += p0; rs1 += p1;
+                pk[i] = tc::pack_bf16(p0, p1);
+            }
+            tc::tmem_st16(lane_addr + kColP + b * (kKeys / 2) + 16, pk);
+            l += rs0 + rs1;
             tc::tmem_st_wait();
             tc::tc_fence_before();
-            tc::mbar_arrive(&bars->p_full);        // P(j) (and any correction of O) is in TMEM
+            tc::mbar_arrive(&bars->p_full[b]);     // P(j) (and any correction of O) is in TMEM
         }
 
         // ---- epilogue: O / l (plus the candidate's own key), or the split partial
-        if (ok && nb > 0) ok = __all_sync(0xffffffffu, tc::mbar_wait(&bars->pv_done, (nb - 1) & 1, err));
+        if (ok && nb > 0) ok = __all_sync(0xffffffffu, tc::mbar_wait(&bars->p_free[(nb - 1) & 1], ((nb - 1) >> 1) & 1, err));
         tc::tc_fence_after();
         if (ok) {
             float o[kDh];

@@ -212,16 +212,16 @@ int Forward::run_t(const CallDesc &call, float *scores, cudaStream_t stream, std
         std::vector<Tile> tiles;
         for (int u = 0; u < B; ++u) {
             const SeqDesc &sd = call.seqs[(size_t)u];
-            const int nPB = (sd.n_paged + 127) / 128, nLB = (sd.n_lin + 127) / 128;
+            const int nPB = (sd.n_paged + 63) / 64, nLB = (sd.n_lin + 63) / 64;      // key blocks of 64 (one page each)
             for (int q0 = 0; q0 < sd.n_q; q0 += 128) {
                 const int n_q = std::min(128, sd.n_q - q0);
                 const int tp1 = sd.q_pos0 + q0 + n_q - 1;
                 const int kmax = tp1 < sd.causal_end ? tp1 : sd.causal_end - 1;      // last key position any row of the tile sees
                 int nb = 0;
                 if (kmax >= 0) {
-                    const int pb = sd.n_paged > 0 ? std::min(nPB, kmax / 128 + 1) : 0;
+                    const int pb = sd.n_paged > 0 ? std::min(nPB, kmax / 64 + 1) : 0;
                     int lb = 0;
-                    if (pb == nPB && sd.n_lin > 0 && kmax >= sd.lin_pos0) lb = std::min(nLB, (kmax - sd.lin_pos0) / 128 + 1);
+                    if (pb == nPB && sd.n_lin > 0 && kmax >= sd.lin_pos0) lb = std::min(nLB, (kmax - sd.lin_pos0) / 64 + 1);
                     nb = pb + lb;
                 }
                 tiles.push_back({u, q0, n_q, nb});
@@ -234,7 +234,7 @@ int Forward::run_t(const CallDesc &call, float *scores, cudaStream_t stream, std
         int part_slot = 0;
         std::sort(tiles.begin(), tiles.end(), [](const Tile &x, const Tile &y) { return x.nb > y.nb; });   // longest first
         for (const Tile &t : tiles) {
-            int ns = std::max(1, std::min(want, t.nb / 4));          // at least 4 key blocks per split
+            int ns = std::max(1, std::min(want, t.nb / 8));          // at least 8 key blocks (512 keys) per split
             if (ns > 1 && part_slot + ns * H > kMaxSplitTiles) ns = 1;
             const bool has_cand = call.seqs[(size_t)t.seq].q_pos0 + t.q0 + t.n_q > call.seqs[(size_t)t.seq].causal_end;
             for (int h = 0; h < H; ++h) {
