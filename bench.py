@@ -29,8 +29,9 @@ METRIC = "candidates ranked/s with cached prefix KV (rank on cache); p50/p99 ran
 UNIT = "candidates/s"
 WORKLOAD = "config2: 4 layers, d_model 256, 4 heads x 64, FFN 1024, bf16; 32 users x (prefix 2048 cached, 64 short-term, 512 candidates); Zipf(1.1) ids over 1M items"
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one attention launch of this workload (ncu; see profiles/)
-ATTENTION_DRAM_TRAFFIC_BYTES = None
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of this workload's rank step, from the ncu captures
+# summarised under profiles/ (None = no capture of the kernel as it stands).
+DRAM_TRAFFIC_BYTES = {"attention": 100.5e6, "gemm": None}
 
 
 def load_peaks():
@@ -245,18 +246,31 @@ def main():
         pool.rank(built.dev_batches[i % nrot], scores)
     prof = B.relaygr_profile_read(model.ctx)
     B.relaygr_profile_enable(model.ctx, False)
-    attn_ms = prof["attention_ms"] / max(1, prof["attention_launches"])
-    attn_flops = workloads.attention_flops_per_layer(shape, built.batches[0], "rank")
     peaks = load_peaks()
-    attn_tflops = attn_flops / (attn_ms * 1e-3) / 1e12
     prof_total = sum(prof[k] for k in prof if k.endswith("_ms"))
+    b0 = built.batches[0]
+    # algorithmic FLOPs of the two tensor-core kernel classes over one rank step (dead last-layer work excluded)
+    attn_flops_step = workloads.batch_flops(shape, b0, "rank") - workloads.batch_linear_flops(shape, b0, "rank")
+    class_flops = {"attention": attn_flops_step, "gemm": workloads.batch_linear_flops(shape, b0, "rank")}
+    class_name = {"attention": "attention_tc_kernel (rank on cache)", "gemm": "gemm_tc_kernel (QKV, out-proj, FFN of the rank step)"}
+    rooflines = {}
+    for cls in ("attention", "gemm"):
+        n_launch = max(1, prof[cls + "_launches"])
+        ms = prof[cls + "_ms"] / n_launch                       # average launch duration, CUDA events on the launching stream
+        fl = class_flops[cls] * prof_steps / n_launch           # algorithmic FLOPs per launch
+        tf = fl / (ms * 1e-3) / 1e12
+        rooflines[cls] = {"kernel": class_name[cls], "bound": "tensor", "achieved": tf, "peak": peaks["tflops"], "unit": "TFLOP/s",
+                          "frac": tf / peaks["tflops"], "peak_source": peaks["source"], "traffic": DRAM_TRAFFIC_BYTES[cls],
+                          "ms_per_launch": ms, "launches_per_step": n_launch / prof_steps, "algorithmic_flops_per_launch": fl,
+                          "share_of_step": prof[cls + "_ms"] / prof_total if prof_total else None}
+    dominant = max(rooflines, key=lambda c: rooflines[c]["share_of_step"] or 0.0)
+    other = "gemm" if dominant == "attention" else "attention"
 
     # ---- end to end through host buffers ------------------------------------------------------------
     hb = [(torch.from_numpy(b.short_ids).pin_memory(), torch.from_numpy(b.cand_ids).pin_memory()) for b in built.batches]
     d_short = torch.empty_like(built.dev_batches[0].short_ids)
     d_cand = torch.empty_like(built.dev_batches[0].cand_ids)
     h_scores = torch.empty(n_cand, dtype=torch.float32).pin_memory()
-    b0 = built.batches[0]
     ctx, kp = model.ctx, pool.pool
 
     def e2e_step(i):
@@ -325,11 +339,7 @@ def main():
             "whole_step_roofline": {"rank_tflops": rank_flops / (ms_per_step * 1e-3) / 1e12,
                                     "rank_frac": rank_flops / (ms_per_step * 1e-3) / 1e12 / peaks["tflops"],
                                     "full_recompute_tflops": full_flops / (float(np.median(full_lat)) * 1e-3) / 1e12},
-            "roofline": {"kernel": "attention_tc_kernel (rank)", "bound": "tensor", "achieved": attn_tflops, "peak": peaks["tflops"],
-                         "unit": "TFLOP/s", "frac": attn_tflops / peaks["tflops"], "peak_source": peaks["source"],
-                         "traffic": ATTENTION_DRAM_TRAFFIC_BYTES, "ms_per_launch": attn_ms,
-                         "algorithmic_flops_per_launch": attn_flops,
-                         "share_of_step": prof["attention_ms"] / prof_total if prof_total else None},
+            "roofline": rooflines[dominant], "roofline_second_kernel": rooflines[other],
             "kernel_ms_per_step": {k: prof[k] / prof_steps for k in prof if k.endswith("_ms")},
             "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks, "cpu_baseline": cpu,
         }

@@ -66,6 +66,24 @@ def attention_flops_per_layer(shape: synth.ModelShape, batch: synth.Batch, mode:
     return tot
 
 
+def batch_linear_flops(shape: synth.ModelShape, batch: synth.Batch, mode: str) -> float:
+    """Algorithmic FLOPs of the linear maps (QKV, out-proj, FFN) of one call: ``batch_flops`` minus attention."""
+    L, d = shape.n_layers, shape.d_model
+    lin = linear_flops_per_token(shape)
+    tot = 0.0
+    for i in range(batch.n_users):
+        P = int(batch.prefix_off[i + 1] - batch.prefix_off[i])
+        S = int(batch.short_off[i + 1] - batch.short_off[i])
+        C = int(batch.cand_off[i + 1] - batch.cand_off[i])
+        if mode == "preinfer":
+            tot += (L - 1) * lin * P + 4.0 * d * d * P
+        elif mode == "rank":
+            tot += (L - 1) * lin * (S + C) + 4.0 * d * d * S + lin * C
+        else:
+            tot += (L - 1) * lin * (P + S + C) + 4.0 * d * d * (P + S) + lin * C
+    return tot
+
+
 def batch_flops(shape: synth.ModelShape, batch: synth.Batch, mode: str) -> float:
     tot = 0.0
     for i in range(batch.n_users):
