@@ -254,6 +254,47 @@ int32_t relaygr_rank_full(relaygr_ctx *ctx, int32_t n_users,
                           float *scores, void *stream);
 
 /*
+ * Full inference for callers that cannot hand the library any scratch memory.  (The paper has
+ * no counterpart: this is a convenience of this library, not a step of the method.)
+ *
+ * Who needs it: code that runs where device allocation is off limits and that holds no
+ * workspace to lend - a serving process whose whole HBM was carved up at start-up and whose
+ * allocator is sealed afterwards, a plug-in running inside another framework's memory pool,
+ * a request handler on a latency-critical thread where cudaMalloc's implicit device
+ * synchronisation is not acceptable.  For them the miss fallback (relaygr_rank_full) would
+ * otherwise be unusable, because that call needs a workspace from relaygr_set_workspace.
+ *
+ * Same arguments, results and errors as relaygr_rank_full, but the scratch (activations,
+ * per-call metadata, split-attention partials, status word) lives in one array of
+ * RELAYGR_STATIC_SCRATCH_BYTES that is part of the library image: every GPU that loads the
+ * library holds that much memory until the process exits, whether or not this call is used.
+ * The call allocates nothing on the device or in pinned memory (it calls no cudaMalloc,
+ * cudaFree or allocating library routine); any workspace lent with relaygr_set_workspace is
+ * neither needed nor touched.
+ *
+ *   - A batch whose scratch need (relaygr_workspace_bytes for its rows, users and zero pages)
+ *     exceeds RELAYGR_STATIC_SCRATCH_BYTES is rejected with RELAYGR_E_NOSPACE and nothing is
+ *     enqueued.  As a guide, one user of a 4-layer d_model-256 bf16 model with a few thousand
+ *     tokens fits; large batches do not - lend a workspace and use relaygr_rank_full.
+ *   - The first call on each device looks the array's device address up and clears its status
+ *     word with a blocking memset; make that first call before any stream capture begins.
+ *     The ctx's device must be the current device.
+ *   - Every call, from every ctx and thread of the process, shares the one array of its
+ *     device, and the array keeps the previous call's contents.  What must start clean is
+ *     cleared on `stream` at the start of each call; two calls whose kernels may overlap on
+ *     the GPU (different streams without an ordering between them) race - order them.
+ *   - If kernels of this call record an internal error, the code is also copied into the
+ *     status word of the ctx's lent workspace, when there is one, so that
+ *     relaygr_device_status reports it.
+ */
+#define RELAYGR_STATIC_SCRATCH_BYTES (96u << 20)
+int32_t relaygr_rank_full_static(relaygr_ctx *ctx, int32_t n_users,
+                                 const int32_t *prefix_ids, const int32_t *prefix_off,
+                                 const int32_t *short_ids, const int32_t *short_off,
+                                 const int32_t *cand_ids, const int32_t *cand_off,
+                                 float *scores, void *stream);
+
+/*
  * Per-kernel timing for benchmarks.  While enabled, every launch of a compute call is
  * bracketed by CUDA events on the call's stream (a few microseconds of overhead per
  * launch: do not leave it on for latency measurements).  relaygr_profile_read waits for

@@ -85,6 +85,7 @@ SIGNATURES = {
     "relaygr_preinfer": (_I32, [_P, _P, _I32, _P, _P, _P, _P]),
     "relaygr_rank": (_I32, [_P, _P, _I32, _P, _P, _P, _P, _P, _P, _P, _P]),
     "relaygr_rank_full": (_I32, [_P, _I32, _P, _P, _P, _P, _P, _P, _P, _P]),
+    "relaygr_rank_full_static": (_I32, [_P, _I32, _P, _P, _P, _P, _P, _P, _P, _P]),
     "relaygr_profile_enable": (_I32, [_P, _I32]),
     "relaygr_profile_read": (_I32, [_P, C.POINTER(Profile)]),
     "relaygr_launch_count": (_I32, [_P, C.POINTER(_I64)]),
@@ -257,6 +258,18 @@ def relaygr_rank_full(ctx, n_users, prefix_ids_dev, prefix_off, short_ids_dev, s
     po, so, co = _host_i32(prefix_off), _host_i32(short_off), _host_i32(cand_off)
     return _check(lib().relaygr_rank_full(ctx, n_users, _ptr(prefix_ids_dev), _ptr(po), _ptr(short_ids_dev), _ptr(so),
                                           _ptr(cand_ids_dev), _ptr(co), _ptr(scores_dev), stream), ok)
+
+
+STATIC_SCRATCH_BYTES = 96 << 20      # RELAYGR_STATIC_SCRATCH_BYTES
+
+
+def relaygr_rank_full_static(ctx, n_users, prefix_ids_dev, prefix_off, short_ids_dev, short_off, cand_ids_dev, cand_off,
+                             scores_dev, stream=None, ok=(OK,)) -> int:
+    """Full inference on the scratch array built into the library: for callers that may not allocate device
+    memory and have no workspace to lend.  Batches beyond the array's size return E_NOSPACE."""
+    po, so, co = _host_i32(prefix_off), _host_i32(short_off), _host_i32(cand_off)
+    return _check(lib().relaygr_rank_full_static(ctx, n_users, _ptr(prefix_ids_dev), _ptr(po), _ptr(short_ids_dev), _ptr(so),
+                                                 _ptr(cand_ids_dev), _ptr(co), _ptr(scores_dev), stream), ok)
 
 
 def relaygr_profile_enable(ctx, on: bool):

@@ -3,6 +3,7 @@
 #include <algorithm>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <string>
 #include <vector>
@@ -457,6 +458,105 @@ int32_t relaygr_rank_full(relaygr_ctx *ctx, int32_t n_users, const int32_t *pref
     rc = ctx->fwd.check_capacity(call, g_err);
     if (rc) return rc;
     return ctx->fwd.run(call, scores, (cudaStream_t)stream, g_err);
+}
+
+// ---- full inference on scratch that is part of the library image ------------------------------------
+
+namespace {
+// The scratch of relaygr_rank_full_static.  In host code this name is only a stand-in for the
+// symbol: the address kernels may use comes from cudaGetSymbolAddress, per device.
+static __device__ __align__(256) unsigned char g_static_scratch[RELAYGR_STATIC_SCRATCH_BYTES];
+
+constexpr int kMaxDevices = 64;
+void *g_static_scratch_addr[kMaxDevices] = {};     // device address of the array, looked up once per device
+std::mutex g_static_scratch_mu;
+
+// Copies a non-zero status word of the static scratch into the ctx's lent workspace, where
+// relaygr_device_status reads it.
+__global__ void forward_status_kernel(const int *from, int *to)
+{
+    const int v = *from;
+    if (v != 0) atomicCAS(to, 0, v);
+}
+
+// Device address of the array on the current device `dev`; the first call per device also clears the status word.
+int static_scratch_address(int dev, void **out)
+{
+    std::lock_guard<std::mutex> lock(g_static_scratch_mu);
+    if (!g_static_scratch_addr[dev]) {
+        void *p = nullptr;
+        cudaError_t e = cudaGetSymbolAddress(&p, g_static_scratch);
+        if (e != cudaSuccess) return fail_cuda("rank_full_static: cudaGetSymbolAddress of the built-in scratch", e);
+        if (!p || ((uintptr_t)p & 255) != 0) return fail(RELAYGR_E_CUDA, "rank_full_static: built-in scratch has no usable device address");
+        e = cudaMemset(p, 0, 1024);
+        if (e != cudaSuccess) return fail_cuda("rank_full_static: clearing the built-in scratch", e);
+        g_static_scratch_addr[dev] = p;
+    }
+    *out = g_static_scratch_addr[dev];
+    return RELAYGR_OK;
+}
+}  // namespace
+
+int32_t relaygr_rank_full_static(relaygr_ctx *ctx, int32_t n_users, const int32_t *prefix_ids, const int32_t *prefix_off,
+                                 const int32_t *short_ids, const int32_t *short_off, const int32_t *cand_ids,
+                                 const int32_t *cand_off, float *scores, void *stream)
+{
+    int rc = need_device(ctx);
+    if (rc) return rc;
+    if (n_users < 0) return fail(RELAYGR_E_INVALID, "bad argument");
+    if (n_users == 0) return RELAYGR_OK;
+    // the same argument checks as relaygr_rank_full, made here first so that a bad call enqueues nothing at all
+    rc = check_offsets(prefix_off, n_users, "prefix", false);
+    if (rc) return rc;
+    rc = check_offsets(short_off, n_users, "short-term", true);
+    if (rc) return rc;
+    rc = check_offsets(cand_off, n_users, "candidate", true);
+    if (rc) return rc;
+    if (!prefix_ids || (short_off[n_users] > 0 && !short_ids) || (cand_off[n_users] > 0 && (!cand_ids || !scores)))
+        return fail(RELAYGR_E_INVALID, "ids / scores pointer is NULL");
+
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return fail_cuda("rank_full_static: cudaGetDevice", e);
+    if (dev != ctx->fwd.device) return fail(RELAYGR_E_INVALID, "rank_full_static: the ctx's device must be the current device");
+    if (dev < 0 || dev >= kMaxDevices) return fail(RELAYGR_E_UNSUPPORTED, "rank_full_static: device ordinal out of range");
+
+    const int64_t rows = (int64_t)prefix_off[n_users] + short_off[n_users] + cand_off[n_users];
+    const size_t need = ctx->fwd.layout(rows, n_users, 0).total;
+    if (need > (size_t)RELAYGR_STATIC_SCRATCH_BYTES) {
+        char msg[256];
+        std::snprintf(msg, sizeof(msg),
+                      "rank_full_static: this batch (%lld token rows, %d users) needs %zu bytes of scratch but the built-in array "
+                      "holds %zu; lend a workspace and call relaygr_rank_full",
+                      (long long)rows, (int)n_users, need, (size_t)RELAYGR_STATIC_SCRATCH_BYTES);
+        return fail(RELAYGR_E_NOSPACE, msg);
+    }
+
+    void *scratch = nullptr;
+    rc = static_scratch_address(dev, &scratch);
+    if (rc) return rc;
+    // the array keeps the last call's contents: the status word must start at zero, everything else is
+    // written before it is read
+    e = cudaMemsetAsync(scratch, 0, 1024, (cudaStream_t)stream);
+    if (e != cudaSuccess) return fail_cuda("rank_full_static: clearing the status word", e);
+
+    // run the ordinary full-inference call with the built-in array standing in for the lent workspace
+    char *lent = ctx->fwd.ws;
+    const size_t lent_bytes = ctx->fwd.ws_bytes;
+    ctx->fwd.ws = (char *)scratch;
+    ctx->fwd.ws_bytes = (size_t)RELAYGR_STATIC_SCRATCH_BYTES;
+    rc = relaygr_rank_full(ctx, n_users, prefix_ids, prefix_off, short_ids, short_off, cand_ids, cand_off, scores, stream);
+    ctx->fwd.ws = lent;
+    ctx->fwd.ws_bytes = lent_bytes;
+    if (rc != RELAYGR_OK) return rc;
+
+    if (lent && lent_bytes >= 1024) {
+        forward_status_kernel<<<1, 1, 0, (cudaStream_t)stream>>>((const int *)scratch, (int *)lent);
+        ctx->fwd.launches += 1;
+        e = cudaGetLastError();
+        if (e != cudaSuccess) return fail_cuda("rank_full_static: status forwarding", e);
+    }
+    return RELAYGR_OK;
 }
 
 }  // extern "C"
