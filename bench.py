@@ -126,8 +126,10 @@ def main():
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--users", type=int, default=32)
-    ap.add_argument("--prefix", type=int, default=2048)
+    ap.add_argument("--workload", type=int, default=2, choices=[2, 3, 4],
+                    help="2 = production-shaped rank (the metric's workload), 3 = jagged batch with shuffled pages, 4 = long-sequence model")
+    ap.add_argument("--users", type=int, default=0, help="0 = the workload's own batch size")
+    ap.add_argument("--prefix", type=int, default=0, help="0 = the workload's own prefix length (2048; 8192 for workload 4)")
     args = ap.parse_args()
     if args.impl == "reference":
         return reference_arm(args)
@@ -149,15 +151,27 @@ def main():
         dist_mod.init_process_group("nccl", device_id=torch.device("cuda", local))
         dist = dist_mod
 
-    wl = synth.workload(2)
+    wl = synth.workload(args.workload)
     shape = wl.model
-    n_users, P, S, C = args.users, args.prefix, 64, 512
+    if args.workload == 3:
+        n_users = args.users or 128
+        pl, sl, cl = synth.config3_lengths(np.random.default_rng(wl.seed + 1000 * rank), n_users)
+        p_lens, s_lens, c_lens = [int(x) for x in pl], [int(x) for x in sl], [int(x) for x in cl]
+        workload_name = "config3: config-2 model; %d users, prefix log-uniform [512, 8192] (sum %d), short U[16,128], candidates U[128,1024] (sum %d); pages scattered by a shuffled page table" % (n_users, sum(p_lens), sum(c_lens))
+    elif args.workload == 4:
+        n_users, P = args.users or 16, args.prefix or 8192
+        p_lens, s_lens, c_lens = [P] * n_users, [128] * n_users, [1024] * n_users
+        workload_name = "config4: 8 layers, d_model 512, 8 heads x 64, FFN 2048, bf16; %d users x (prefix %d cached, 128 short-term, 1024 candidates)" % (n_users, P)
+    else:
+        n_users, P = args.users or 32, args.prefix or 2048
+        p_lens, s_lens, c_lens = [P] * n_users, [64] * n_users, [512] * n_users
+        workload_name = WORKLOAD if (n_users, P) == (32, 2048) else "config2 model; %d users x (prefix %d cached, 64 short-term, 512 candidates)" % (n_users, P)
     # replicas: every rank holds its own users (user-hash placement), no data-path collective
-    built = workloads.build(shape, wl.seed + 1000 * rank, [P] * n_users, [S] * n_users, [C] * n_users, n_rotations=8,
+    built = workloads.build(shape, wl.seed + 1000 * rank, p_lens, s_lens, c_lens, n_rotations=8, shuffle_pages=args.workload == 3,
                             first_user=rank * n_users, device="cuda:%d" % local)
     model, pool = built.model, built.pool
     stream = torch.cuda.current_stream()
-    n_cand = n_users * C
+    n_cand = int(sum(c_lens))
     scores = torch.empty(n_cand, dtype=torch.float32, device=model.device)
 
     def barrier():
@@ -260,7 +274,7 @@ def main():
         fl = class_flops[cls] * prof_steps / n_launch           # algorithmic FLOPs per launch
         tf = fl / (ms * 1e-3) / 1e12
         rooflines[cls] = {"kernel": class_name[cls], "bound": "tensor", "achieved": tf, "peak": peaks["tflops"], "unit": "TFLOP/s",
-                          "frac": tf / peaks["tflops"], "peak_source": peaks["source"], "traffic": DRAM_TRAFFIC_BYTES[cls],
+                          "frac": tf / peaks["tflops"], "peak_source": peaks["source"], "traffic": DRAM_TRAFFIC_BYTES[cls] if workload_name == WORKLOAD else None,
                           "ms_per_launch": ms, "launches_per_step": n_launch / prof_steps, "algorithmic_flops_per_launch": fl,
                           "share_of_step": prof[cls + "_ms"] / prof_total if prof_total else None}
     dominant = max(rooflines, key=lambda c: rooflines[c]["share_of_step"] or 0.0)
@@ -298,7 +312,7 @@ def main():
 
     # ---- CPU baseline: the checker, timed on this machine's host cores ----------------------------------
     cpu = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+    if rank == 0 and world == 1 and not args.no_cpu_baseline and args.workload == 2:
         from oracle import ref
         om = ref.Model(shape.n_layers, shape.d_model, shape.n_heads, shape.d_head, shape.d_ff, shape.ln_eps,
                        {**built.weights.mat, **built.weights.vec})
@@ -314,7 +328,7 @@ def main():
             want = om.rank_cached(K, V, s, c)
             t_cpu += time.perf_counter() - t0
             err = max(err, float(np.max(np.abs(got[b0.cand_off[u]:b0.cand_off[u + 1]] - want))))
-        cpu = {"value": n_sample * C / t_cpu, "unit": UNIT, "cores": ref.n_threads(), "kind": "oracle",
+        cpu = {"value": n_sample * c_lens[0] / t_cpu, "unit": UNIT, "cores": ref.n_threads(), "kind": "oracle",
                "sample": "%d of the %d users of one batch, rank on cache only (prefix K/V from the checker's own pre-infer, untimed)" % (n_sample, n_users),
                "max_abs_err_vs_gpu": err}
 
@@ -326,15 +340,15 @@ def main():
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": WORKLOAD, "step": "one relaygr_rank call over the batch, prefix KV already in the paged pool",
-                       "users": n_users, "prefix": P, "short": S, "candidates": C,
-                       "l2": "inputs larger than L2: each step streams %.0f MiB of prefix K/V and rotates 8 input sets" % (n_users * shape.kv_bytes(P) / 2**20),
+            "config": {"workload": workload_name, "step": "one relaygr_rank call over the batch, prefix KV already in the paged pool",
+                       "users": n_users, "prefix_tokens": int(sum(p_lens)), "short_tokens": int(sum(s_lens)), "candidates": n_cand,
+                       "l2": "inputs larger than L2: each step streams %.0f MiB of prefix K/V and rotates 8 input sets" % (shape.kv_bytes(int(sum(p_lens))) / 2**20),
                        "parallelism": "replicas (users hashed to GPUs), no collective" if world > 1 else "single GPU"},
             "latency_ms": {"rank_p50_backlogged": float(np.percentile(lat, 50)), "rank_p99_backlogged": float(np.percentile(lat, 99)),
                            "rank_p50": float(np.percentile(lat1, 50)), "rank_p99": float(np.percentile(lat1, 99)),
                            "full_recompute_p50": float(np.percentile(full_lat, 50)), "full_recompute_p99": float(np.percentile(full_lat, 99)),
                            "rank_beats_full_recompute_p99": bool(np.percentile(lat1, 99) < np.percentile(full_lat, 99))},
-            "preinfer": {"tokens_per_s": n_users * P / (pre_ms_med * 1e-3), "ms": pre_ms_med,
+            "preinfer": {"tokens_per_s": int(sum(p_lens)) / (pre_ms_med * 1e-3), "ms": pre_ms_med,
                          "frac_of_tensor_roofline": pre_flops / (pre_ms_med * 1e-3) / 1e12 / peaks["tflops"]},
             "whole_step_roofline": {"rank_tflops": rank_flops / (ms_per_step * 1e-3) / 1e12,
                                     "rank_frac": rank_flops / (ms_per_step * 1e-3) / 1e12 / peaks["tflops"],
