@@ -239,3 +239,42 @@ def test_spill_and_reload_round_trip_is_bit_exact():
         assert torch.equal(k0, k1) and torch.equal(v0, v1)
     assert model.device_status() == 0
     pool.close(); model.close()
+
+
+# ---------------------------------------------------------------- full-size workloads, sampled users against the checker
+def _full_size(workload_index, p_lens, s_lens, c_lens, sample, shuffle):
+    """Runs pre-infer + rank + full inference at the sizes and launch configuration the benchmark times, and
+    checks the scores of the sampled users (every candidate of theirs) against the checker."""
+    from paper_2601_01712_b200 import workloads
+    wl = synth.workload(workload_index)
+    built = workloads.build(wl.model, wl.seed, p_lens, s_lens, c_lens, n_rotations=1, shuffle_pages=shuffle)
+    b, db = built.batches[0], built.dev_batches[0]
+    built.pool.preinfer(db)
+    scores = built.pool.rank(db).cpu().numpy()
+    full = built.model.rank_full(db).cpu().numpy()
+    assert built.model.device_status() == 0
+    assert np.all(np.isfinite(scores)) and np.all(np.isfinite(full))
+    # property that holds at any size: rank on cache and full inference agree (the paper's relation)
+    assert np.max(np.abs(scores - full)) <= TOL_BF16
+    om = oracle_model(wl.model, built.weights)
+    want = oracle_scores(om, b, users=sample)
+    assert max_abs_err(scores, b, want) <= TOL_BF16
+    assert max_abs_err(full, b, want) <= TOL_BF16
+    built.pool.close(); built.model.close()
+
+
+def test_config2_full_size_sampled_users():
+    _full_size(2, [2048] * 32, [64] * 32, [512] * 32, sample=[0, 13, 31], shuffle=False)
+
+
+def test_config3_jagged_full_size_sampled_users():
+    wl = synth.workload(3)
+    p, s, c = synth.config3_lengths(np.random.default_rng(wl.seed), 128)
+    p, s, c = [int(x) for x in p], [int(x) for x in s], [int(x) for x in c]
+    order = np.argsort(p)
+    sample = [int(order[0]), int(order[40]), int(order[90])]        # a short, a middling and a long prefix
+    _full_size(3, p, s, c, sample=sample, shuffle=True)
+
+
+def test_config4_long_model_sampled_user():
+    _full_size(4, [4096] * 16, [128] * 16, [1024] * 16, sample=[5], shuffle=False)
