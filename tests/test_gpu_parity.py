@@ -278,3 +278,37 @@ def test_config3_jagged_full_size_sampled_users():
 
 def test_config4_long_model_sampled_user():
     _full_size(4, [4096] * 16, [128] * 16, [1024] * 16, sample=[5], shuffle=False)
+
+
+def test_reload_tier_workload_small():
+    """The reload-tier workload at a reduced population: every call's scores equal those of the same users ranked
+    from prefixes that never left HBM (bit for bit: spill and reload move bytes), and the tiers are accounted for."""
+    from paper_2601_01712_b200 import tier_workload
+    B, rt = _runtime()
+    shape = small_bf16_shape()
+    report, kept, (model, pool, w, rotations) = tier_workload.run(
+        population=48, hbm_users=12, prefix=300, batch=8, n_short=9, n_cand=40, calls=25, warmup=3, shape=shape, collect_scores=True)
+    assert report["reloads"] > 0 and report["hit_rate"]["host"] > 0 and report["hit_rate"]["hbm"] > 0
+    assert report["spilled_at_start"] == 48 and report["pcie_gb_per_s"] > 0
+    pool.close()
+    # reference: a pool large enough for everybody, same seeded prefixes (the workload draws them first, in user order)
+    rng = np.random.default_rng(synth.BASE_SEED + 5)
+    zipf = synth.ZipfIds(shape.vocab, 1.1)
+    big = rt.KvPool(model, 48 * synth.pages_for(300))
+    for u0 in range(0, 48, 8):
+        users = np.arange(u0, u0 + 8, dtype=np.uint64)
+        b = synth.make_batch(zipf, rng, [300] * 8, [0] * 8, [0] * 8)
+        b.users = users
+        for u in users:
+            big.alloc(int(u), 300)
+        big.preinfer(rt.DeviceBatch(b, model.device))
+    so, co = np.arange(9, dtype=np.int32) * 9, np.arange(9, dtype=np.int32) * 40
+    for users, rot, got in kept[3:]:
+        sid, cid = rotations[rot]
+        want = torch.empty(8 * 40, dtype=torch.float32, device=model.device)
+        B.relaygr_rank(model.ctx, big.pool, users, sid.data_ptr(), so, cid.data_ptr(), co, want.data_ptr(),
+                       torch.cuda.current_stream().cuda_stream)
+        torch.cuda.synchronize()
+        assert torch.equal(got, want)
+    assert model.device_status() == 0
+    big.close(); model.close()
