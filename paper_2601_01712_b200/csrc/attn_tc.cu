@@ -11,9 +11,11 @@
 //     O += P V    tcgen05.mma M=128 N=64 K=64, A = P from TMEM, B = V in shared memory (MN-major),
 //                 O accumulated in TMEM
 // S and P are double-buffered in TMEM, so the MMA warp runs one block ahead of the softmax and
-// the tensor pipe never waits for it in steady state.  The running maximum is only raised (and
-// O rescaled in TMEM, after the pending PV has drained) when it grows by more than 2^8, which
-// keeps every exponent in range and makes the rescale rare.
+// the tensor pipe never waits for it in steady state.  The exponentials of a block are taken
+// against the running maximum as it stood before the block; only when the block's row sum shows
+// that some exponent may have exceeded 2^8 is the block maximum computed, the running maximum
+// raised, O rescaled in TMEM (after the pending PV has drained) and the block redone - so no
+// maximum is on the fast path, every exponent that is kept stays below 2^8, and rescales are rare.
 //
 // Warp roles (192 threads): warp 0 = TMA producer, warp 1 = TMEM owner + MMA issuer,
 // warps 2-5 = softmax / correction / epilogue (TMEM lane quadrant = warp index % 4).
@@ -32,7 +34,7 @@ constexpr int kStagesKV = 4;
 constexpr int kSmemBytes = kQBytes + 2 * kStagesKV * kKVBytes + 1024 + 512;
 constexpr uint32_t kTmemCols = 256;                 // S[2]: 0..127, P[2]: 128..191, O: 192..255
 constexpr uint32_t kColS = 0, kColP = 128, kColO = 192;
-constexpr float kRescaleThreshold = 8.f;            // in log2 units
+constexpr float kRowSumLimit = 256.f;               // a block's row sum above this: some p may exceed 2^8 -> redo against a raised maximum
 
 struct Bars {
     uint64_t q_full;
@@ -129,8 +131,9 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             }
         }
     } else if (warp == 1) {
-        // ---------------------------------------------------------------- MMA issuer
-        if (lane == 0) {
+        // ---------------------------------------------------------------- MMA issuer (the whole warp walks the loop so
+        // that addresses and descriptors stay warp-uniform; one elected lane issues the tcgen05 instructions)
+        {
             constexpr uint32_t idesc_qk = tc::make_idesc(128, kKeys, 0, 0);   // Q, K both K-major
             constexpr uint32_t idesc_pv = tc::make_idesc(128, kDh, 0, 1);     // P from TMEM, V MN-major
             const uint64_t qdesc = tc::smem_desc_sw128(tc::smem_u32(sQ));
@@ -141,11 +144,14 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 if (j >= 2 && !tc::mbar_wait(&bars->s_free[b], ((j >> 1) - 1) & 1, err)) return false;
                 tc::tc_fence_after();
                 const uint64_t kdesc = tc::smem_desc_sw128(tc::smem_u32(sK + s * kKVBytes));
+                if (tc::elect_one()) {
 #pragma unroll
-                for (int k = 0; k < kDh / 16; ++k)
-                    tc::mma_ss(tmem_base + kColS + b * kKeys, qdesc + 2 * k, kdesc + 2 * k, idesc_qk, k != 0);
-                tc::mma_commit(&bars->s_full[b]);
-                tc::mma_commit(&bars->k_empty[s]);
+                    for (int k = 0; k < kDh / 16; ++k)
+                        tc::mma_ss(tmem_base + kColS + b * kKeys, qdesc + 2 * k, kdesc + 2 * k, idesc_qk, k != 0);
+                    tc::mma_commit(&bars->s_full[b]);
+                    tc::mma_commit(&bars->k_empty[s]);
+                }
+                __syncwarp();
                 return true;
             };
             if (ok && nb > 0) ok = issue_qk(0);
@@ -156,11 +162,16 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 if (!tc::mbar_wait(&bars->v_full[s], (j / kStagesKV) & 1, err)) break;
                 tc::tc_fence_after();
                 const uint64_t vdesc = tc::smem_desc_sw128(tc::smem_u32(sV + s * kKVBytes));
+                if (tc::elect_one()) {
 #pragma unroll
-                for (int k = 0; k < kKeys / 16; ++k)      // 16 keys per instruction: 8 TMEM columns of P, 2048 bytes of V
-                    tc::mma_ts(tmem_base + kColO, tmem_base + kColP + b * (kKeys / 2) + 8 * k, vdesc + 128 * k, idesc_pv, (j | k) != 0);
-                tc::mma_commit(&bars->p_free[b]);          // P[b] consumed; also "O holds blocks 0..j"
-                tc::mma_commit(&bars->v_empty[s]);
+                    for (int k = 0; k < kKeys / 16; ++k)      // 16 keys per instruction: 8 TMEM columns of P, 2048 bytes of V
+                        tc::mma_ts(tmem_base + kColO, tmem_base + kColP + b * (kKeys / 2) + 8 * k, vdesc + 128 * k, idesc_pv, (j | k) != 0);
+                    tc::mma_commit(&bars->p_free[b]);          // P[b] consumed; also "O holds blocks 0..j"
+                    tc::mma_commit(&bars->v_empty[s]);
+                }
+                __syncwarp();
+                // QK(j + 2) follows PV(j) in issue order, and a commit covers everything issued before it: a softmax
+                // thread that sees s_full of block j + 2 also knows that P[b] has been consumed
                 if (j + 2 < nb) ok = issue_qk(j + 2);      // S[b] was freed by the softmax of block j
             }
         }
@@ -204,59 +215,70 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     if (32 + i >= jmax) s1[i] = 0xff800000u;
                 }
             }
-            float mx = -INFINITY;
+            // p = 2^(s c - m c), bf16 P into TMEM (P[b] is free: see the MMA issuer), row sum in fp32.  The exponentials
+            // are first taken against the running maximum as it stood before this block; only if the row sum shows that
+            // some p may have exceeded 2^8 (or the row has no maximum yet) is the block maximum computed, the running
+            // maximum raised, O rescaled and the block redone.  No maximum is on the fast path.
+            auto exp_block = [&](float mc) {
+                float r0 = 0.f, r1 = 0.f, r2 = 0.f, r3 = 0.f;
+                uint32_t pk[16];
 #pragma unroll
-            for (int i = 0; i < 32; i += 2) {
-                mx = max3(mx, __uint_as_float(s0[i]), __uint_as_float(s0[i + 1]));
-                mx = max3(mx, __uint_as_float(s1[i]), __uint_as_float(s1[i + 1]));
-            }
-            // raise the running maximum only when it grows by more than the threshold
-            float alpha = 1.f;
-            const bool raise = (mx - m) * c > kRescaleThreshold;    // false when mx == -inf; true on the first visible key
-            if (raise) {
-                alpha = (m == -INFINITY) ? 0.f : ex2((m - mx) * c);
-                m = mx;
-            }
-            const float mc = (m == -INFINITY) ? 0.f : m * c;
-            if (j > 0 && __any_sync(0xffffffffu, raise)) {
-                // correction: O must hold blocks 0..j-1 completely before it is rescaled
-                ok = __all_sync(0xffffffffu, tc::mbar_wait(&bars->p_free[(j - 1) & 1], ((j - 1) >> 1) & 1, err));
-                if (!ok) break;
-                tc::tc_fence_after();
-#pragma unroll 1
-                for (int cc = 0; cc < kDh; cc += 16) {
-                    uint32_t ov[16];
-                    tc::tmem_ld16(lane_addr + kColO + cc, ov);
-                    tc::tmem_ld_wait();
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) ov[i] = __float_as_uint(__uint_as_float(ov[i]) * alpha);
-                    tc::tmem_st16(lane_addr + kColO + cc, ov);
+                for (int i = 0; i < 16; i += 2) {
+                    const float p0 = ex2(fmaf(__uint_as_float(s0[2 * i]), c, -mc)), p1 = ex2(fmaf(__uint_as_float(s0[2 * i + 1]), c, -mc));
+                    const float p2 = ex2(fmaf(__uint_as_float(s0[2 * i + 2]), c, -mc)), p3 = ex2(fmaf(__uint_as_float(s0[2 * i + 3]), c, -mc));
+                    r0 += p0; r1 += p1; r2 += p2; r3 += p3;
+                    pk[i] = tc::pack_bf16(p0, p1); pk[i + 1] = tc::pack_bf16(p2, p3);
                 }
-            }
-            l *= alpha;
-            // P[b] was last read by the PV of block j - 2
-            if (j >= 2) {
-                ok = __all_sync(0xffffffffu, tc::mbar_wait(&bars->p_free[b], ((j >> 1) - 1) & 1, err));
-                if (!ok) break;
-            }
-            // p = 2^(s c - m c); row sum in fp32; bf16 P into TMEM
-            float rs0 = 0.f, rs1 = 0.f;
-            uint32_t pk[16];
+                tc::tmem_st16(lane_addr + kColP + b * (kKeys / 2), pk);
 #pragma unroll
-            for (int i = 0; i < 16; ++i) {
-                const float p0 = ex2(fmaf(__uint_as_float(s0[2 * i]), c, -mc)), p1 = ex2(fmaf(__uint_as_float(s0[2 * i + 1]), c, -mc));
-                rs0 += p0; rs1 += p1;
-                pk[i] = tc::pack_bf16(p0, p1);
+                for (int i = 0; i < 16; i += 2) {
+                    const float p0 = ex2(fmaf(__uint_as_float(s1[2 * i]), c, -mc)), p1 = ex2(fmaf(__uint_as_float(s1[2 * i + 1]), c, -mc));
+                    const float p2 = ex2(fmaf(__uint_as_float(s1[2 * i + 2]), c, -mc)), p3 = ex2(fmaf(__uint_as_float(s1[2 * i + 3]), c, -mc));
+                    r0 += p0; r1 += p1; r2 += p2; r3 += p3;
+                    pk[i] = tc::pack_bf16(p0, p1); pk[i + 1] = tc::pack_bf16(p2, p3);
+                }
+                tc::tmem_st16(lane_addr + kColP + b * (kKeys / 2) + 16, pk);
+                return (r0 + r1) + (r2 + r3);
+            };
+            float rs = 0.f, alpha = 1.f;
+            bool redo = true;
+            if (j > 0) {
+                rs = exp_block((m == -INFINITY) ? 0.f : m * c);
+                redo = __any_sync(0xffffffffu, !(rs <= kRowSumLimit) || m == -INFINITY);
             }
-            tc::tmem_st16(lane_addr + kColP + b * (kKeys / 2), pk);
+            if (redo) {
+                float mx = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
 #pragma unroll
-            for (int i = 0; i < 16; ++i) {
-                const float p0 = ex2(fmaf(__uint_as_float(s1[2 * i]), c, -mc)), p1 = ex2(fmaf(__uint_as_float(s1[2 * i + 1]), c, -mc));
-                rs0 += p0; rs1 += p1;
-                pk[i] = tc::pack_bf16(p0, p1);
+                for (int i = 0; i < 32; i += 4) {
+                    mx = max3(mx, __uint_as_float(s0[i]), __uint_as_float(s0[i + 1]));
+                    mx1 = max3(mx1, __uint_as_float(s0[i + 2]), __uint_as_float(s0[i + 3]));
+                    mx2 = max3(mx2, __uint_as_float(s1[i]), __uint_as_float(s1[i + 1]));
+                    mx3 = max3(mx3, __uint_as_float(s1[i + 2]), __uint_as_float(s1[i + 3]));
+                }
+                mx = fmaxf(fmaxf(mx, mx1), fmaxf(mx2, mx3));
+                const bool raise = mx > m;                    // false when mx == -inf
+                if (raise) {
+                    alpha = (m == -INFINITY) ? 0.f : ex2((m - mx) * c);
+                    m = mx;
+                }
+                if (j > 0 && __any_sync(0xffffffffu, raise)) {
+                    // correction: O must hold blocks 0..j-1 completely before it is rescaled
+                    ok = __all_sync(0xffffffffu, tc::mbar_wait(&bars->p_free[(j - 1) & 1], ((j - 1) >> 1) & 1, err));
+                    if (!ok) break;
+                    tc::tc_fence_after();
+#pragma unroll 1
+                    for (int cc = 0; cc < kDh; cc += 16) {
+                        uint32_t ov[16];
+                        tc::tmem_ld16(lane_addr + kColO + cc, ov);
+                        tc::tmem_ld_wait();
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) ov[i] = __float_as_uint(__uint_as_float(ov[i]) * alpha);
+                        tc::tmem_st16(lane_addr + kColO + cc, ov);
+                    }
+                }
+                rs = exp_block((m == -INFINITY) ? 0.f : m * c);
             }
-            tc::tmem_st16(lane_addr + kColP + b * (kKeys / 2) + 16, pk);
-            l += rs0 + rs1;
+            l = fmaf(l, alpha, rs);
             tc::tmem_st_wait();
             tc::tc_fence_before();
             tc::mbar_arrive(&bars->p_full[b]);     // P(j) (and any correction of O) is in TMEM
