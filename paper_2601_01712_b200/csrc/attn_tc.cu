@@ -50,6 +50,26 @@ __device__ __forceinline__ float ex2(float x)
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
+// Packed pairs of fp32 (sm_100 executes fma / add on two lanes of a 64-bit register per instruction).
+__device__ __forceinline__ uint64_t pack2(float lo, float hi)
+{
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float &lo, float &hi) { asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v)); }
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c)
+{
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b)
+{
+    uint64_t d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
 __device__ __forceinline__ float max3(float a, float b, float c)
 {
     float d;
@@ -220,25 +240,32 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             // some p may have exceeded 2^8 (or the row has no maximum yet) is the block maximum computed, the running
             // maximum raised, O rescaled and the block redone.  No maximum is on the fast path.
             auto exp_block = [&](float mc) {
-                float r0 = 0.f, r1 = 0.f, r2 = 0.f, r3 = 0.f;
+                const uint64_t c2 = pack2(c, c), nmc2 = pack2(-mc, -mc);
+                uint64_t ra = pack2(0.f, 0.f), rb = ra;
                 uint32_t pk[16];
 #pragma unroll
                 for (int i = 0; i < 16; i += 2) {
-                    const float p0 = ex2(fmaf(__uint_as_float(s0[2 * i]), c, -mc)), p1 = ex2(fmaf(__uint_as_float(s0[2 * i + 1]), c, -mc));
-                    const float p2 = ex2(fmaf(__uint_as_float(s0[2 * i + 2]), c, -mc)), p3 = ex2(fmaf(__uint_as_float(s0[2 * i + 3]), c, -mc));
-                    r0 += p0; r1 += p1; r2 += p2; r3 += p3;
+                    float x0, x1, x2, x3;
+                    unpack2(fma2(pack2(__uint_as_float(s0[2 * i]), __uint_as_float(s0[2 * i + 1])), c2, nmc2), x0, x1);
+                    unpack2(fma2(pack2(__uint_as_float(s0[2 * i + 2]), __uint_as_float(s0[2 * i + 3])), c2, nmc2), x2, x3);
+                    const float p0 = ex2(x0), p1 = ex2(x1), p2 = ex2(x2), p3 = ex2(x3);
+                    ra = add2(ra, pack2(p0, p1)); rb = add2(rb, pack2(p2, p3));
                     pk[i] = tc::pack_bf16(p0, p1); pk[i + 1] = tc::pack_bf16(p2, p3);
                 }
                 tc::tmem_st16(lane_addr + kColP + b * (kKeys / 2), pk);
 #pragma unroll
                 for (int i = 0; i < 16; i += 2) {
-                    const float p0 = ex2(fmaf(__uint_as_float(s1[2 * i]), c, -mc)), p1 = ex2(fmaf(__uint_as_float(s1[2 * i + 1]), c, -mc));
-                    const float p2 = ex2(fmaf(__uint_as_float(s1[2 * i + 2]), c, -mc)), p3 = ex2(fmaf(__uint_as_float(s1[2 * i + 3]), c, -mc));
-                    r0 += p0; r1 += p1; r2 += p2; r3 += p3;
+                    float x0, x1, x2, x3;
+                    unpack2(fma2(pack2(__uint_as_float(s1[2 * i]), __uint_as_float(s1[2 * i + 1])), c2, nmc2), x0, x1);
+                    unpack2(fma2(pack2(__uint_as_float(s1[2 * i + 2]), __uint_as_float(s1[2 * i + 3])), c2, nmc2), x2, x3);
+                    const float p0 = ex2(x0), p1 = ex2(x1), p2 = ex2(x2), p3 = ex2(x3);
+                    ra = add2(ra, pack2(p0, p1)); rb = add2(rb, pack2(p2, p3));
                     pk[i] = tc::pack_bf16(p0, p1); pk[i + 1] = tc::pack_bf16(p2, p3);
                 }
                 tc::tmem_st16(lane_addr + kColP + b * (kKeys / 2) + 16, pk);
-                return (r0 + r1) + (r2 + r3);
+                float r0, r1;
+                unpack2(add2(ra, rb), r0, r1);
+                return r0 + r1;
             };
             float rs = 0.f, alpha = 1.f;
             bool redo = true;
