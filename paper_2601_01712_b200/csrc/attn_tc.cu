@@ -92,15 +92,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     Bars *bars = reinterpret_cast<Bars *>(sV + kStagesKV * kKVBytes);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const AttnItem it = items[blockIdx.x];
-    const SeqDesc sd = seqs[it.seq];
-    const int nb = it.blk1 - it.blk0;
-    const int n_paged_blocks = (sd.n_paged + kKeys - 1) / kKeys;      // = the user's page count
-
-    if (threadIdx.x == 0) bars->abort_flag = *reinterpret_cast<volatile int *>(err);
-    __syncthreads();
-    if (bars->abort_flag != 0) return;
-
+    // set-up that touches nothing earlier kernels wrote; it may run while the previous kernel is still finishing
     if (threadIdx.x == 0) {
         tc::mbar_init(&bars->q_full, 1);
         for (int s = 0; s < kStagesKV; ++s) {
@@ -118,12 +110,21 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         tc::tmem_alloc(&bars->tmem_slot, kTmemCols);
         tc::tmem_relinquish();
     }
+    grid_launch_dependents();
+    grid_dependency_wait();                                       // from here on: data of earlier kernels
+    if (threadIdx.x == 0) bars->abort_flag = *reinterpret_cast<volatile int *>(err);
     tc::tc_fence_before();
     __syncthreads();
     tc::tc_fence_after();
     const uint32_t tmem_base = bars->tmem_slot;
+    const bool live = bars->abort_flag == 0;                      // an earlier kernel gave up: do not pile on
+    const AttnItem it = items[blockIdx.x];
+    const SeqDesc sd = seqs[it.seq];
+    const int nb = it.blk1 - it.blk0;
+    const int n_paged_blocks = (sd.n_paged + kKeys - 1) / kKeys;      // = the user's page count
 
-    if (warp == 0) {
+    if (!live) {
+    } else if (warp == 0) {
         // ---------------------------------------------------------------- TMA producer
         if (lane == 0) {
             tc::mbar_expect_tx(&bars->q_full, kQBytes);
@@ -397,6 +398,8 @@ __global__ void __launch_bounds__(128)
 attention_merge_kernel(const AttnMerge *__restrict__ merges, const SeqDesc *__restrict__ seqs, const float *__restrict__ partial,
                        int d_model, __nv_bfloat16 *__restrict__ out)
 {
+    grid_launch_dependents();
+    grid_dependency_wait();
     const AttnMerge mg = merges[blockIdx.x];
     const int r = threadIdx.x;
     if (r >= mg.n_q) return;
@@ -437,14 +440,12 @@ cudaError_t launch_attention_tc(const CUtensorMap &tmQ, const CUtensorMap &tmK, 
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
-    attention_tc_kernel<<<n_items, 192, kSmemBytes, stream>>>(tmQ, tmK, tmV, tmPool, items, seqs, pt, n_layers, layer, d_model, q,
-                                                              k_lin, v_lin, out, partial, err);
     *launches += 1;
-    cudaError_t e = cudaGetLastError();
+    cudaError_t e = launch_dependent(attention_tc_kernel, dim3(n_items), dim3(192), (size_t)kSmemBytes, stream, tmQ, tmK, tmV, tmPool, items,
+                                     seqs, pt, n_layers, layer, d_model, q, k_lin, v_lin, out, partial, err);
     if (e != cudaSuccess || n_merges == 0) return e;
-    attention_merge_kernel<<<n_merges, 128, 0, stream>>>(merges, seqs, partial, d_model, out);
     *launches += 1;
-    return cudaGetLastError();
+    return launch_dependent(attention_merge_kernel, dim3(n_merges), dim3(128), 0, stream, merges, seqs, partial, d_model, out);
 }
 
 }  // namespace relaygr

@@ -136,10 +136,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int n_tiles_n = N / BN;
     const int64_t n_tiles = ((M + BM - 1) / BM) * n_tiles_n;
 
-    if (threadIdx.x == 0) bars->abort_flag = *reinterpret_cast<volatile int *>(err);
-    __syncthreads();
-    if (bars->abort_flag != 0) return;                            // an earlier kernel gave up: do not pile on
-
+    // set-up that touches nothing earlier kernels wrote; it may run while the previous kernel is still finishing
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { tc::mbar_init(&bars->full[s], 1); tc::mbar_init(&bars->empty[s], 1); }
         for (int s = 0; s < 2; ++s) { tc::mbar_init(&bars->acc_full[s], 1); tc::mbar_init(&bars->acc_empty[s], kEpiWarps); }
@@ -151,12 +148,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         tc::tmem_alloc(&bars->tmem_slot, kTmemCols);
         tc::tmem_relinquish();
     }
+    grid_launch_dependents();
+    grid_dependency_wait();                                       // from here on: data of earlier kernels
+    if (threadIdx.x == 0) bars->abort_flag = *reinterpret_cast<volatile int *>(err);
     tc::tc_fence_before();
     __syncthreads();
     tc::tc_fence_after();
     const uint32_t tmem_base = bars->tmem_slot;
+    const bool live = bars->abort_flag == 0;                      // an earlier kernel gave up: do not pile on
 
-    if (warp == 0) {
+    if (!live) {
+    } else if (warp == 0) {
         // ---------------------------------------------------------------- TMA producer
         if (lane == 0) {
             uint32_t it = 0;
@@ -282,9 +284,8 @@ cudaError_t launch_gemm_tc(const CUtensorMap &tmA, const CUtensorMap &tmB, int64
     }
     const int64_t tiles = ((M + BM - 1) / BM) * (N / BN);
     const unsigned grid = (unsigned)(tiles < n_sms ? tiles : n_sms);
-    gemm_tc_kernel<<<grid, kThreads, kSmemBytes, stream>>>(tmA, tmB, M, N, K, epi, err);
     *launches += 1;
-    return cudaGetLastError();
+    return launch_dependent(gemm_tc_kernel, dim3(grid), dim3(kThreads), (size_t)kSmemBytes, stream, tmA, tmB, M, N, K, epi, err);
 }
 
 }  // namespace relaygr

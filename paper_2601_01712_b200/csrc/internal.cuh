@@ -73,6 +73,13 @@ struct Epilogue {
     int32_t n_users;
 };
 
+// Programmatic dependent launch: a kernel launched with launch_dependent() may start while the kernel before it on
+// the stream is still running.  It does its set-up (barriers, TMEM, descriptor prefetch), then calls
+// grid_dependency_wait() before it touches anything that earlier kernels wrote; grid_launch_dependents() lets the
+// kernel after it start its own set-up as soon as every CTA of this one has begun.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 __device__ __forceinline__ int find_user(const int32_t *row_off, int n_users, int row)
 {
     // largest u with row_off[u] <= row

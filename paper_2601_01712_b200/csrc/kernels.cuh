@@ -4,9 +4,25 @@
 
 #include <cuda.h>
 
+#include <utility>
+
 #include "internal.cuh"
 
 namespace relaygr {
+
+// Launch with programmatic stream serialisation: the kernel may begin before its predecessor on the stream has
+// finished, and must call grid_dependency_wait() before reading or writing what earlier kernels produce.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, Args &&...args)
+{
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
 
 // ---- memory-bound steps (CUDA cores, vectorised loads, warp-shuffle reductions) ----------------
 

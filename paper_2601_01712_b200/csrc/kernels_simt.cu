@@ -102,6 +102,8 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32)
 gather_ln_kernel(const T *__restrict__ emb, int64_t vocab, int d, RowSource src, int64_t n_rows,
                  const float *__restrict__ g, const float *__restrict__ b, float eps, float *__restrict__ x, T *__restrict__ a)
 {
+    grid_launch_dependents();
+    grid_dependency_wait();
     const int64_t row = (int64_t)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     if (row >= n_rows) return;
@@ -120,21 +122,61 @@ gather_ln_kernel(const T *__restrict__ emb, int64_t vocab, int d, RowSource src,
     ln_row_store<T>(v, d, lane, g, b, eps, a + row * d);
 }
 
-template <typename T>
+// a[r, :] = LN(x[r, :]).  A warp takes ROWS consecutive rows at once and issues all their loads before any
+// arithmetic, so that enough bytes are in flight per SM to reach HBM / L2 bandwidth; NC = chunks of 128 columns.
+template <typename T, int NC, int ROWS>
 __global__ void __launch_bounds__(kWarpsPerBlock * 32)
 layernorm_kernel(const float *__restrict__ x, int d, int64_t n_rows, const float *__restrict__ g, const float *__restrict__ b,
                  float eps, T *__restrict__ a)
 {
-    const int64_t row = (int64_t)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
+    grid_launch_dependents();
+    grid_dependency_wait();
+    const int64_t row0 = ((int64_t)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5)) * ROWS;
     const int lane = threadIdx.x & 31;
-    if (row >= n_rows) return;
-    float4 v[kMaxChunks];
+    if (row0 >= n_rows) return;
+    float4 v[ROWS][NC];
 #pragma unroll
-    for (int c = 0; c < kMaxChunks; ++c) {
+    for (int r = 0; r < ROWS; ++r)
+#pragma unroll
+        for (int c = 0; c < NC; ++c) {
+            const int i = (c * 32 + lane) * 4;
+            v[r][c] = (row0 + r < n_rows && i < d) ? load4(x + (row0 + r) * d + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+    float4 gg[NC], bb[NC];
+#pragma unroll
+    for (int c = 0; c < NC; ++c) {
         const int i = (c * 32 + lane) * 4;
-        if (i < d) v[c] = load4(x + row * d + i);
+        if (i < d) { gg[c] = load4(g + i); bb[c] = load4(b + i); }
     }
-    ln_row_store<T>(v, d, lane, g, b, eps, a + row * d);
+    const float inv_d = 1.f / (float)d;
+#pragma unroll
+    for (int r = 0; r < ROWS; ++r) {
+        if (row0 + r >= n_rows) break;
+        float s = 0.f;
+#pragma unroll
+        for (int c = 0; c < NC; ++c) s += (v[r][c].x + v[r][c].y) + (v[r][c].z + v[r][c].w);      // padding chunks hold zeros
+        const float mean = warp_sum(s) * inv_d;
+        float q = 0.f;
+#pragma unroll
+        for (int c = 0; c < NC; ++c)
+            if ((c * 32 + lane) * 4 < d) {
+                const float a0 = v[r][c].x - mean, a1 = v[r][c].y - mean, a2 = v[r][c].z - mean, a3 = v[r][c].w - mean;
+                q += a0 * a0 + a1 * a1 + a2 * a2 + a3 * a3;
+            }
+        const float rstd = rsqrtf(warp_sum(q) * inv_d + eps);
+#pragma unroll
+        for (int c = 0; c < NC; ++c) {
+            const int i = (c * 32 + lane) * 4;
+            if (i < d) {
+                float4 o;
+                o.x = (v[r][c].x - mean) * rstd * gg[c].x + bb[c].x;
+                o.y = (v[r][c].y - mean) * rstd * gg[c].y + bb[c].y;
+                o.z = (v[r][c].z - mean) * rstd * gg[c].z + bb[c].z;
+                o.w = (v[r][c].w - mean) * rstd * gg[c].w + bb[c].w;
+                store4(a + (row0 + r) * d + i, o);
+            }
+        }
+    }
 }
 
 __global__ void __launch_bounds__(kWarpsPerBlock * 32)
@@ -142,6 +184,8 @@ score_kernel(const float *__restrict__ x, int d, const SeqDesc *__restrict__ seq
              const int32_t *__restrict__ score_off, const float *__restrict__ g, const float *__restrict__ b, float eps,
              const float *__restrict__ w, const float *__restrict__ bias, float *__restrict__ scores)
 {
+    grid_launch_dependents();
+    grid_dependency_wait();
     const int64_t idx = (int64_t)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     if (idx >= n_total) return;
@@ -337,9 +381,9 @@ cudaError_t launch_gather_ln(const T *emb, int64_t vocab, int d, RowSource src, 
                              const float *b, float eps, float *x, T *a, cudaStream_t stream, int64_t *launches)
 {
     if (n_rows == 0) return cudaSuccess;
-    gather_ln_kernel<T><<<blocks_for(n_rows), kWarpsPerBlock * 32, 0, stream>>>(emb, vocab, d, src, n_rows, g, b, eps, x, a);
     *launches += 1;
-    return cudaGetLastError();
+    return launch_dependent(gather_ln_kernel<T>, dim3(blocks_for(n_rows)), dim3(kWarpsPerBlock * 32), 0, stream, emb, vocab, d, src, n_rows, g,
+                            b, eps, x, a);
 }
 
 template <typename T>
@@ -347,9 +391,18 @@ cudaError_t launch_layernorm(const float *x, int d, int64_t n_rows, const float 
                              cudaStream_t stream, int64_t *launches)
 {
     if (n_rows == 0) return cudaSuccess;
-    layernorm_kernel<T><<<blocks_for(n_rows), kWarpsPerBlock * 32, 0, stream>>>(x, d, n_rows, g, b, eps, a);
+    const int nc = (d + 127) / 128;
+    cudaError_t e;
+#define RELAYGR_LN(NC, ROWS)                                                                                              \
+    e = launch_dependent(layernorm_kernel<T, NC, ROWS>, dim3(blocks_for((n_rows + ROWS - 1) / ROWS)), dim3(kWarpsPerBlock * 32), 0, stream, \
+                         x, d, n_rows, g, b, eps, a)
+    if (nc <= 1) RELAYGR_LN(1, 4);
+    else if (nc <= 2) RELAYGR_LN(2, 4);
+    else if (nc <= 4) RELAYGR_LN(4, 2);
+    else RELAYGR_LN(8, 1);
+#undef RELAYGR_LN
     *launches += 1;
-    return cudaGetLastError();
+    return e;
 }
 
 cudaError_t launch_score(const float *x, int d, const SeqDesc *seqs, int n_users, int64_t n_total, const int32_t *score_off,
@@ -357,10 +410,9 @@ cudaError_t launch_score(const float *x, int d, const SeqDesc *seqs, int n_users
                          cudaStream_t stream, int64_t *launches)
 {
     if (n_total == 0) return cudaSuccess;
-    score_kernel<<<blocks_for(n_total), kWarpsPerBlock * 32, 0, stream>>>(x, d, seqs, n_users, n_total, score_off, g, b, eps,
-                                                                         w, bias, scores);
     *launches += 1;
-    return cudaGetLastError();
+    return launch_dependent(score_kernel, dim3(blocks_for(n_total)), dim3(kWarpsPerBlock * 32), 0, stream, x, d, seqs, n_users, n_total,
+                            score_off, g, b, eps, w, bias, scores);
 }
 
 template <typename T>
