@@ -394,35 +394,35 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
 }
 
 // Combine the (m, l, O) partials of a split work item:  O = sum_i 2^((m_i - M) c) O_i / sum_i 2^((m_i - M) c) l_i.
-__global__ void __launch_bounds__(128)
+// blockIdx.x = item, blockIdx.y = group of 8 rows; one warp per row, a lane per pair of output columns: every load is a
+// coalesced row segment and all rows are in flight at once (the kernel is a chain of two memory round trips).
+__global__ void __launch_bounds__(256)
 attention_merge_kernel(const AttnMerge *__restrict__ merges, const SeqDesc *__restrict__ seqs, const float *__restrict__ partial,
                        int d_model, __nv_bfloat16 *__restrict__ out)
 {
     grid_launch_dependents();
     grid_dependency_wait();
     const AttnMerge mg = merges[blockIdx.x];
-    const int r = threadIdx.x;
-    if (r >= mg.n_q) return;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const float c = 0.125f * 1.4426950408889634f;
-    float M = -INFINITY;
-    for (int i = 0; i < mg.n_splits; ++i) M = fmaxf(M, partial[((size_t)(mg.slot0 + i) * kQTile + r) * (kDh + 2)]);
-    float o[kDh];
-#pragma unroll
-    for (int e = 0; e < kDh; ++e) o[e] = 0.f;
-    float l = 0.f;
-    for (int i = 0; i < mg.n_splits; ++i) {
-        const float *p = partial + ((size_t)(mg.slot0 + i) * kQTile + r) * (kDh + 2);
-        const float mi = p[0];
-        const float wgt = (mi == -INFINITY) ? 0.f : ex2((mi - M) * c);
-        l = fmaf(p[1], wgt, l);
-#pragma unroll
-        for (int e = 0; e < kDh; ++e) o[e] = fmaf(p[2 + e], wgt, o[e]);
+    const int64_t row0 = (int64_t)seqs[mg.seq].q_row0 + mg.q0;
+    const int r = blockIdx.y * 8 + warp;
+    if (r < mg.n_q) {
+        float M = -INFINITY;
+        for (int i = 0; i < mg.n_splits; ++i) M = fmaxf(M, partial[((size_t)(mg.slot0 + i) * kQTile + r) * (kDh + 2)]);
+        float o0 = 0.f, o1 = 0.f, l = 0.f;
+        for (int i = 0; i < mg.n_splits; ++i) {
+            const float *p = partial + ((size_t)(mg.slot0 + i) * kQTile + r) * (kDh + 2);
+            const float mi = p[0];
+            const float wgt = (mi == -INFINITY) ? 0.f : ex2((mi - M) * c);
+            const float2 v = *reinterpret_cast<const float2 *>(p + 2 + 2 * lane);
+            l = fmaf(p[1], wgt, l);
+            o0 = fmaf(v.x, wgt, o0);
+            o1 = fmaf(v.y, wgt, o1);
+        }
+        const float inv = 1.f / l;
+        *reinterpret_cast<uint32_t *>(out + (row0 + r) * d_model + mg.head * kDh + 2 * lane) = tc::pack_bf16(o0 * inv, o1 * inv);
     }
-    const float inv = 1.f / l;
-    const int64_t row = (int64_t)seqs[mg.seq].q_row0 + mg.q0 + r;
-    __nv_bfloat16 *dst = out + row * d_model + mg.head * kDh;
-#pragma unroll
-    for (int e = 0; e < kDh; e += 2) *reinterpret_cast<uint32_t *>(dst + e) = tc::pack_bf16(o[e] * inv, o[e + 1] * inv);
 }
 
 }  // namespace
@@ -445,7 +445,7 @@ cudaError_t launch_attention_tc(const CUtensorMap &tmQ, const CUtensorMap &tmK, 
                                      seqs, pt, n_layers, layer, d_model, q, k_lin, v_lin, out, partial, err);
     if (e != cudaSuccess || n_merges == 0) return e;
     *launches += 1;
-    return launch_dependent(attention_merge_kernel, dim3(n_merges), dim3(128), 0, stream, merges, seqs, partial, d_model, out);
+    return launch_dependent(attention_merge_kernel, dim3(n_merges, kQTile / 8), dim3(256), 0, stream, merges, seqs, partial, d_model, out);
 }
 
 }  // namespace relaygr
