@@ -139,7 +139,7 @@ def main():
     from paper_2601_01712_b200 import build as libbuild
     libbuild.build()
     from paper_2601_01712_b200 import binding as B
-    from paper_2601_01712_b200 import synth, workloads
+    from paper_2601_01712_b200 import replicas, synth, workloads
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -180,11 +180,7 @@ def main():
         torch.cuda.synchronize()
 
     def max_over_ranks(ms):
-        if dist is None:
-            return ms
-        t = torch.tensor([ms], dtype=torch.float64, device=model.device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+        return replicas.max_over_ranks(ms, dist, model.device)
 
     # ---- pre-infer (timed beside the metric) --------------------------------------------------------
     pre_steps = max(3, min(20, args.steps // 20))
