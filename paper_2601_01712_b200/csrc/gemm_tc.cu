@@ -20,18 +20,25 @@ namespace relaygr {
 
 namespace {
 
-constexpr int BM = 128, BN = 128, BK = 64, STAGES = 4;
+constexpr int BM = 128, BK = 64, kMaxStages = 4;
 constexpr int kEpiWarps = 8;
 constexpr int kThreads = 32 * (2 + kEpiWarps);
-constexpr int kABytes = BM * BK * 2, kBBytes = BN * BK * 2, kStage = kABytes + kBBytes;
+constexpr int kABytes = BM * BK * 2;
 constexpr int kPatchPitchF32 = 36;                                  // floats per staged row (32 + 4 pad): conflict-free float4 access
 constexpr int kPatchBytes = 32 * kPatchPitchF32 * 4;                // 4608 B per warp
-constexpr int kSmemBytes = STAGES * kStage + kEpiWarps * kPatchBytes + kEpiWarps * 32 * 8 /*row offsets*/ + 256 /*barriers*/ +
-                           1024 /*alignment slack*/;
-constexpr uint32_t kTmemCols = 2 * BN;
+
+// Tile width BN: 128, or 256 for long mainloops (gemm_tile_n).  The stage ring is as deep as shared memory allows.
+template <int BN> struct Cfg {
+    static constexpr int kBBytes = BN * BK * 2;
+    static constexpr int kStage = kABytes + kBBytes;
+    static constexpr int kStages = BN == 256 ? 3 : 4;
+    static constexpr int kSmemBytes = kStages * kStage + kEpiWarps * kPatchBytes + kEpiWarps * 32 * 8 /*row offsets*/ + 256 /*barriers*/ +
+                                      1024 /*alignment slack*/;
+    static constexpr uint32_t kTmemCols = 2 * BN;
+};
 
 struct GemmBars {
-    uint64_t full[STAGES], empty[STAGES];
+    uint64_t full[kMaxStages], empty[kMaxStages];
     uint64_t acc_full[2], acc_empty[2];
     uint32_t tmem_slot;
     int abort_flag;
@@ -121,10 +128,13 @@ __device__ __forceinline__ void epilogue_chunk(const Epilogue &e, int64_t m_base
     __syncwarp();
 }
 
+template <int BN>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, int64_t M, int N, int K,
                Epilogue epi, int *err)
 {
+    constexpr int STAGES = Cfg<BN>::kStages, kStage = Cfg<BN>::kStage;
+    constexpr uint32_t kTmemCols = Cfg<BN>::kTmemCols;
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     float *patches = reinterpret_cast<float *>(smem + STAGES * kStage);
@@ -177,8 +187,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             }
         }
     } else if (warp == 1) {
-        // ---------------------------------------------------------------- MMA issuer
-        if (lane == 0) {
+        // ---------------------------------------------------------------- MMA issuer (the whole warp walks the loop so that
+        // addresses stay warp-uniform; one elected lane issues the tcgen05 instructions)
+        {
             constexpr uint32_t idesc = tc::make_idesc(BM, BN, 0, 0);
             uint32_t it = 0, ti = 0;
             bool ok = true;
@@ -194,19 +205,23 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     tc::tc_fence_after();
                     const uint32_t a = tc::smem_u32(smem + s * kStage);
                     const uint64_t adesc = tc::smem_desc_sw128(a), bdesc = tc::smem_desc_sw128(a + kABytes);
+                    if (tc::elect_one()) {
 #pragma unroll
-                    for (int k = 0; k < BK / 16; ++k)     // 32 bytes of K per instruction: descriptor start address + 2
-                        tc::mma_ss(tmem_base + as * BN, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0);
-                    tc::mma_commit(&bars->empty[s]);       // frees the stage when these MMAs have read it
+                        for (int k = 0; k < BK / 16; ++k)     // 32 bytes of K per instruction: descriptor start address + 2
+                            tc::mma_ss(tmem_base + as * BN, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0);
+                        tc::mma_commit(&bars->empty[s]);       // frees the stage when these MMAs have read it
+                        if (kb == kblocks - 1) tc::mma_commit(&bars->acc_full[as]);
+                    }
+                    __syncwarp();
                 }
-                if (ok) tc::mma_commit(&bars->acc_full[as]);
             }
         }
     } else {
         // ---------------------------------------------------------------- epilogue
         const int ew = warp - 2;
         const int quad = warp & 3;                          // TMEM lanes this warp may touch: 32*quad .. 32*quad+31
-        const int half = ew >> 2;                           // columns 64*half .. 64*half+63 of the tile
+        const int half = ew >> 2;                           // columns (BN/2)*half .. +BN/2-1 of the tile, 64 at a time
+        constexpr int kColsPerWarp = BN / 2;
         float *patch = patches + ew * (kPatchBytes / 4);
         int64_t *rowoff = rowoffs + ew * 32;
         const bool scatter = epi.mode == EPI_QKV && epi.paged.slab != nullptr;
@@ -220,7 +235,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const int64_t m = m_base + lane;
             // K / V rows of a pre-infer call go straight into the user's pages: offset of (page, K, slot) per row
             int last_slot = -1, page = 0;
-            if (scatter && epi.col0 + n0 + half * 64 + 63 >= epi.d_model) {
+            if (scatter && epi.col0 + n0 + half * kColsPerWarp + kColsPerWarp - 1 >= epi.d_model) {
                 int64_t off = 0;
                 if (m < M) {
                     const int u = find_user(epi.row_off, epi.n_users, (int)m);
@@ -235,29 +250,34 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             ok = __all_sync(0xffffffffu, tc::mbar_wait(&bars->acc_full[as], (ti >> 1) & 1, err));
             if (!ok) break;
             tc::tc_fence_after();
-            const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + as * BN + half * 64;
-            uint32_t r0[32], r1[32];
-            tc::tmem_ld32(taddr, r0);
-            tc::tmem_ld32(taddr + 32, r1);
-            tc::tmem_ld_wait();
-            tc::tc_fence_before();
-            __syncwarp();
-            if (lane == 0) tc::mbar_arrive(&bars->acc_empty[as]);      // this warp's part of the accumulator is in registers
-            float v[32];
+            const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + as * BN + half * kColsPerWarp;
+#pragma unroll 1
+            for (int pass = 0; pass < kColsPerWarp / 64; ++pass) {
+                uint32_t r0[32], r1[32];
+                tc::tmem_ld32(taddr + pass * 64, r0);
+                tc::tmem_ld32(taddr + pass * 64 + 32, r1);
+                tc::tmem_ld_wait();
+                if (pass == kColsPerWarp / 64 - 1) {
+                    tc::tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) tc::mbar_arrive(&bars->acc_empty[as]);      // this warp's part of the accumulator is in registers
+                }
+                float v[32];
 #pragma unroll
-            for (int cc = 0; cc < 2; ++cc) {
+                for (int cc = 0; cc < 2; ++cc) {
 #pragma unroll
-                for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(cc == 0 ? r0[i] : r1[i]);
-                const int n = n0 + half * 64 + cc * 32;
-                epilogue_chunk(epi, m_base, M, n, N, v, lane, patch, rowoff);
-                if (last_slot >= 0 && last_slot < 63 && epi.col0 + n >= epi.d_model) {
-                    // last prefix row of a user: clear the unused slots of its last page (they are masked, but must hold finite values)
-                    const int col = epi.col0 + n, which = col / epi.d_model, c = col - which * epi.d_model;
-                    __nv_bfloat16 *slab = reinterpret_cast<__nv_bfloat16 *>(epi.paged.slab);
-                    const uint4 z = make_uint4(0, 0, 0, 0);
-                    for (int s = last_slot + 1; s < 64; ++s) {
-                        uint4 *zp = reinterpret_cast<uint4 *>(slab + page_elem_offset(epi.paged, page, which - 1, s) + c);
-                        zp[0] = z; zp[1] = z; zp[2] = z; zp[3] = z;
+                    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(cc == 0 ? r0[i] : r1[i]);
+                    const int n = n0 + half * kColsPerWarp + pass * 64 + cc * 32;
+                    epilogue_chunk(epi, m_base, M, n, N, v, lane, patch, rowoff);
+                    if (last_slot >= 0 && last_slot < 63 && epi.col0 + n >= epi.d_model) {
+                        // last prefix row of a user: clear the unused slots of its last page (they are masked, but must hold finite values)
+                        const int col = epi.col0 + n, which = col / epi.d_model, c = col - which * epi.d_model;
+                        __nv_bfloat16 *slab = reinterpret_cast<__nv_bfloat16 *>(epi.paged.slab);
+                        const uint4 z = make_uint4(0, 0, 0, 0);
+                        for (int s = last_slot + 1; s < 64; ++s) {
+                            uint4 *zp = reinterpret_cast<uint4 *>(slab + page_elem_offset(epi.paged, page, which - 1, s) + c);
+                            zp[0] = z; zp[1] = z; zp[2] = z; zp[3] = z;
+                        }
                     }
                 }
             }
@@ -270,22 +290,29 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
 }  // namespace
 
-cudaError_t launch_gemm_tc(const CUtensorMap &tmA, const CUtensorMap &tmB, int64_t M, int N, int K, const Epilogue &epi,
-                           int *err, cudaStream_t stream, int64_t *launches)
+template <int BN>
+static cudaError_t launch_bn(const CUtensorMap &tmA, const CUtensorMap &tmB, int64_t M, int N, int K, const Epilogue &epi, int *err,
+                             cudaStream_t stream)
 {
-    if (M == 0 || N == 0) return cudaSuccess;
     static int n_sms = 0;
     if (n_sms == 0) {
         int dev = 0;
         cudaError_t e = cudaGetDevice(&dev);
         if (e == cudaSuccess) e = cudaDeviceGetAttribute(&n_sms, cudaDevAttrMultiProcessorCount, dev);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_tc_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<BN>::kSmemBytes);
         if (e != cudaSuccess) { n_sms = 0; return e; }
     }
     const int64_t tiles = ((M + BM - 1) / BM) * (N / BN);
     const unsigned grid = (unsigned)(tiles < n_sms ? tiles : n_sms);
+    return launch_dependent(gemm_tc_kernel<BN>, dim3(grid), dim3(kThreads), (size_t)Cfg<BN>::kSmemBytes, stream, tmA, tmB, M, N, K, epi, err);
+}
+
+cudaError_t launch_gemm_tc(const CUtensorMap &tmA, const CUtensorMap &tmB, int64_t M, int N, int K, const Epilogue &epi,
+                           int *err, cudaStream_t stream, int64_t *launches)
+{
+    if (M == 0 || N == 0) return cudaSuccess;
     *launches += 1;
-    return launch_dependent(gemm_tc_kernel, dim3(grid), dim3(kThreads), (size_t)kSmemBytes, stream, tmA, tmB, M, N, K, epi, err);
+    return gemm_tile_n(N, K) == 256 ? launch_bn<256>(tmA, tmB, M, N, K, epi, err, stream) : launch_bn<128>(tmA, tmB, M, N, K, epi, err, stream);
 }
 
 }  // namespace relaygr

@@ -62,8 +62,13 @@ cudaError_t launch_attention_simt(const T *q, const T *k_lin, const T *v_lin, Pa
 
 // ---- tensor-core kernels (the bf16 model) -------------------------------------------------------------
 
+// Output tile width of the tensor-core GEMM for [*, K] x [N, K]^T (N % 128 == 0): 256 pays only when the mainloop is
+// long (K >= 1024: twice the MMA work per pipeline hand-shake, A read once per 256 columns); with the short K of the
+// other projections the longer epilogue of a wide tile costs more than that gains (measured).
+inline int gemm_tile_n(int N, int K) { return (N % 256 == 0 && K >= 1024) ? 256 : 128; }
+
 // C[m, n] = sum_k A[m, k] W[n, k] on tcgen05; tmA covers A [M, K] with a 128-row box, tmB covers W [N, K]
-// with a 128-row box, both 64 columns wide with the 128-byte swizzle.  N % 128 == 0, K % 64 == 0.
+// with a box of gemm_tile_n(N, K) rows, both 64 columns wide with the 128-byte swizzle.  N % 128 == 0, K % 64 == 0.
 // err is a device status word: kernels record a code there instead of hanging or trapping.
 cudaError_t launch_gemm_tc(const CUtensorMap &tmA, const CUtensorMap &tmB, int64_t M, int N, int K, const Epilogue &epi,
                            int *err, cudaStream_t stream, int64_t *launches);
