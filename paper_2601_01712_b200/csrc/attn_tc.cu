@@ -39,7 +39,7 @@ constexpr float kRowSumLimit = 256.f;               // a block's row sum above t
 struct Bars {
     uint64_t q_full;
     uint64_t k_full[kStagesKV], k_empty[kStagesKV], v_full[kStagesKV], v_empty[kStagesKV];
-    uint64_t s_full[2], s_free[2], p_full[2], p_free[2];
+    uint64_t s_full[2], p_full[2], p_free[2];
     uint32_t tmem_slot;
     int abort_flag;
 };
@@ -100,7 +100,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             tc::mbar_init(&bars->v_full[s], 1); tc::mbar_init(&bars->v_empty[s], 1);
         }
         for (int b = 0; b < 2; ++b) {
-            tc::mbar_init(&bars->s_full[b], 1); tc::mbar_init(&bars->s_free[b], 128);
+            tc::mbar_init(&bars->s_full[b], 1);
             tc::mbar_init(&bars->p_full[b], 128); tc::mbar_init(&bars->p_free[b], 1);
         }
         tc::fence_mbar_init();
@@ -162,7 +162,6 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             auto issue_qk = [&](int j) {        // S[j & 1] = Q K(j)^T
                 const int s = j % kStagesKV, b = j & 1;
                 if (!tc::mbar_wait(&bars->k_full[s], (j / kStagesKV) & 1, err)) return false;
-                if (j >= 2 && !tc::mbar_wait(&bars->s_free[b], ((j >> 1) - 1) & 1, err)) return false;
                 tc::tc_fence_after();
                 const uint64_t kdesc = tc::smem_desc_sw128(tc::smem_u32(sK + s * kKVBytes));
                 if (tc::elect_one()) {
@@ -192,8 +191,9 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 }
                 __syncwarp();
                 // QK(j + 2) follows PV(j) in issue order, and a commit covers everything issued before it: a softmax
-                // thread that sees s_full of block j + 2 also knows that P[b] has been consumed
-                if (j + 2 < nb) ok = issue_qk(j + 2);      // S[b] was freed by the softmax of block j
+                // thread that sees s_full of block j + 2 also knows that P[b] has been consumed.  S[b] is free as well:
+                // P(j) was published only after the softmax had taken S(j) into registers.
+                if (j + 2 < nb) ok = issue_qk(j + 2);
             }
         }
     } else {
@@ -226,9 +226,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             uint32_t s0[32], s1[32];
             tc::tmem_ld32(lane_addr + kColS + b * kKeys, s0);
             tc::tmem_ld32(lane_addr + kColS + b * kKeys + 32, s1);
-            tc::tmem_ld_wait();
-            tc::tc_fence_before();
-            tc::mbar_arrive(&bars->s_free[b]);               // S[b] may be overwritten by the QK^T of block j + 2
+            tc::tmem_ld_wait();                              // (S[b] is handed back with P(j): see the MMA issuer)
             if (need_mask) {
 #pragma unroll
                 for (int i = 0; i < 32; ++i) {
