@@ -35,6 +35,12 @@
  *   - A ctx (and a pool) must not be used from two host threads at once.
  *     Calls on one ctx share its workspace: calls on different streams must
  *     be ordered by the caller.
+ *   - Model slots (Section 3.2, "Concurrency inside a special instance"): several
+ *     ctx created with the same shape and the same weight pointers, each with its
+ *     own workspace, may use ONE pool, e.g. pre-infer of some users on one stream
+ *     while another ctx ranks other users on a second stream.  The pool orders
+ *     producers, consumers, spills and reloads of a user's pages across streams
+ *     with events; the host calls themselves must still come from one thread at a time.
  */
 #ifndef RELAYGR_H_
 #define RELAYGR_H_

@@ -187,6 +187,9 @@ int32_t relaygr_kv_pool_create(relaygr_ctx *ctx, void *hbm_slab, size_t hbm_byte
     relaygr_kv_page_bytes(ctx, &pb);
     if (hbm_bytes < pb) return fail(RELAYGR_E_NOSPACE, "hbm_bytes holds less than one page");
     if (hbm_bytes / pb > (size_t)1 << 24) return fail(RELAYGR_E_UNSUPPORTED, "more than 2^24 pages");
+    // the kernels address the slab as rows of d_model elements through one tensor map with 32-bit row coordinates
+    if ((hbm_bytes / pb) * (size_t)ctx->fwd.cfg.n_layers * 128 >= ((size_t)1 << 31))
+        return fail(RELAYGR_E_UNSUPPORTED, "pool too large: pages * n_layers * 128 must stay below 2^31 (use several pools)");
     relaygr_kv_pool *p = new (std::nothrow) relaygr_kv_pool();
     if (!p) return fail(RELAYGR_E_NOSPACE, "out of host memory");
     p->ctx = ctx;
@@ -281,6 +284,15 @@ int32_t relaygr_kv_stats(relaygr_kv_pool *pool, relaygr_pool_stats *out)
 
 // ---- hot path --------------------------------------------------------------------------------------
 
+// A pool may serve every ctx of the same model (model slots); what matters is that pages mean the same thing.
+static bool same_model(const relaygr_ctx *a, const relaygr_ctx *b)
+{
+    const relaygr_model_cfg &x = a->fwd.cfg, &y = b->fwd.cfg;
+    return a == b || (x.n_layers == y.n_layers && x.d_model == y.d_model && x.n_heads == y.n_heads && x.d_head == y.d_head &&
+                      x.d_ff == y.d_ff && x.dtype == y.dtype && x.page_tokens == y.page_tokens && x.vocab == y.vocab &&
+                      a->host_only == b->host_only && a->fwd.w.w_qkv == b->fwd.w.w_qkv && a->fwd.w.emb == b->fwd.w.emb);
+}
+
 static int need_device(relaygr_ctx *ctx)
 {
     if (!ctx) return fail(RELAYGR_E_INVALID, "ctx is NULL");
@@ -312,7 +324,7 @@ int32_t relaygr_preinfer(relaygr_ctx *ctx, relaygr_kv_pool *pool, int32_t n_user
 {
     int rc = need_device(ctx);
     if (rc) return rc;
-    if (!pool || pool->ctx != ctx) return fail(RELAYGR_E_INVALID, "pool does not belong to this ctx");
+    if (!pool || !same_model(pool->ctx, ctx)) return fail(RELAYGR_E_INVALID, "pool was created for a different model");
     if (n_users < 0 || (n_users > 0 && (!users || !prefix_ids))) return fail(RELAYGR_E_INVALID, "bad argument");
     if (n_users == 0) return RELAYGR_OK;
     rc = check_offsets(prefix_off, n_users, "prefix", false);
@@ -362,7 +374,7 @@ int32_t relaygr_rank(relaygr_ctx *ctx, relaygr_kv_pool *pool, int32_t n_users, c
 {
     int rc = need_device(ctx);
     if (rc) return rc;
-    if (!pool || pool->ctx != ctx) return fail(RELAYGR_E_INVALID, "pool does not belong to this ctx");
+    if (!pool || !same_model(pool->ctx, ctx)) return fail(RELAYGR_E_INVALID, "pool was created for a different model");
     if (n_users < 0 || (n_users > 0 && !users)) return fail(RELAYGR_E_INVALID, "bad argument");
     if (n_users == 0) return RELAYGR_OK;
     rc = check_offsets(short_off, n_users, "short-term", true);

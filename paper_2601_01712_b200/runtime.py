@@ -46,6 +46,15 @@ class Model:
         self._ws = None
         self.page_bytes = B.relaygr_kv_page_bytes(self.ctx)
 
+    def new_slot(self) -> "Model":
+        """Another context on the same weights (a model slot): its own workspace, usable with the same pool."""
+        other = object.__new__(Model)
+        other.shape, other.device, other._t, other.cfg, other._w = self.shape, self.device, self._t, self.cfg, self._w
+        other.ctx = B.relaygr_create(self.cfg, self._w)
+        other._ws = None
+        other.page_bytes = self.page_bytes
+        return other
+
     @property
     def torch_dtype(self):
         return torch.bfloat16 if self.shape.dtype == synth.DTYPE_BF16 else torch.float32
@@ -135,14 +144,15 @@ class KvPool:
     def stats(self):
         return B.relaygr_kv_stats(self.pool)
 
-    def preinfer(self, batch: DeviceBatch, stream=None, ok=(B.OK,)):
-        return B.relaygr_preinfer(self.model.ctx, self.pool, batch.users, batch.prefix_ids.data_ptr(), batch.prefix_off,
+    def preinfer(self, batch: DeviceBatch, stream=None, ok=(B.OK,), slot: Optional[Model] = None):
+        return B.relaygr_preinfer((slot or self.model).ctx, self.pool, batch.users, batch.prefix_ids.data_ptr(), batch.prefix_off,
                                   _stream_ptr(stream), ok)
 
-    def rank(self, batch: DeviceBatch, scores: Optional[torch.Tensor] = None, stream=None, per_user_status=None, ok=(B.OK,)):
+    def rank(self, batch: DeviceBatch, scores: Optional[torch.Tensor] = None, stream=None, per_user_status=None, ok=(B.OK,),
+             slot: Optional[Model] = None):
         if scores is None:
             scores = torch.empty(max(1, int(batch.cand_off[-1])), dtype=torch.float32, device=self.model.device)
-        code = B.relaygr_rank(self.model.ctx, self.pool, batch.users, batch.short_ids.data_ptr(), batch.short_off,
+        code = B.relaygr_rank((slot or self.model).ctx, self.pool, batch.users, batch.short_ids.data_ptr(), batch.short_off,
                               batch.cand_ids.data_ptr(), batch.cand_off, scores.data_ptr(), _stream_ptr(stream),
                               per_user_status, ok)
         return scores[:int(batch.cand_off[-1])] if code == B.OK else None

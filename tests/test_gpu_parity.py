@@ -312,3 +312,16 @@ def test_reload_tier_workload_small():
         assert torch.equal(got, want)
     assert model.device_status() == 0
     big.close(); model.close()
+
+
+def test_two_model_slots_share_one_pool():
+    """Rank by one context while another context pre-infers other users into the same pool, on two streams: the
+    ranked scores are those of an undisturbed run, bit for bit, and match the checker."""
+    from paper_2601_01712_b200 import slots_workload
+    shape = small_bf16_shape()
+    report, scores, batch, w = slots_workload.run(n_rank_users=3, prefix=300, n_short=9, n_cand=40, bg_users=2, bg_prefix=700, calls=12,
+                                                  warmup=2, shape=shape, return_scores=True)
+    assert report["scores_identical_with_and_without_background"]
+    assert report["background_preinfer_calls"] >= 1
+    om = oracle_model(shape, w)
+    assert max_abs_err(scores, batch, oracle_scores(om, batch)) <= TOL_BF16
