@@ -130,6 +130,9 @@ def main():
                     help="2 = production-shaped rank (the metric's workload), 3 = jagged batch with shuffled pages, 4 = long-sequence model")
     ap.add_argument("--users", type=int, default=0, help="0 = the workload's own batch size")
     ap.add_argument("--prefix", type=int, default=0, help="0 = the workload's own prefix length (2048; 8192 for workload 4)")
+    ap.add_argument("--candidates", type=int, default=0, help="candidates per user (0 = the workload's own: 512, or 1024 for workload 4)")
+    ap.add_argument("--layers", type=int, default=0, help="override the model's depth (sweeps)")
+    ap.add_argument("--d-model", type=int, default=0, help="override the model's width (heads of 64, FFN 4x; sweeps)")
     args = ap.parse_args()
     if args.impl == "reference":
         return reference_arm(args)
@@ -153,6 +156,10 @@ def main():
 
     wl = synth.workload(args.workload)
     shape = wl.model
+    if args.layers or args.d_model:
+        dm = args.d_model or shape.d_model
+        shape = synth.ModelShape(args.layers or shape.n_layers, dm, dm // 64, 64, 4 * dm, shape.vocab, shape.dtype)
+    custom = ("; overrides: layers %d, d_model %d" % (shape.n_layers, shape.d_model)) if (args.layers or args.d_model) else ""
     if args.workload == 3:
         n_users = args.users or 128
         pl, sl, cl = synth.config3_lengths(np.random.default_rng(wl.seed + 1000 * rank), n_users)
@@ -160,12 +167,15 @@ def main():
         workload_name = "config3: config-2 model; %d users, prefix log-uniform [512, 8192] (sum %d), short U[16,128], candidates U[128,1024] (sum %d); pages scattered by a shuffled page table" % (n_users, sum(p_lens), sum(c_lens))
     elif args.workload == 4:
         n_users, P = args.users or 16, args.prefix or 8192
-        p_lens, s_lens, c_lens = [P] * n_users, [128] * n_users, [1024] * n_users
-        workload_name = "config4: 8 layers, d_model 512, 8 heads x 64, FFN 2048, bf16; %d users x (prefix %d cached, 128 short-term, 1024 candidates)" % (n_users, P)
+        C = args.candidates or 1024
+        p_lens, s_lens, c_lens = [P] * n_users, [128] * n_users, [C] * n_users
+        workload_name = "config4: 8 layers, d_model 512, 8 heads x 64, FFN 2048, bf16; %d users x (prefix %d cached, 128 short-term, %d candidates)%s" % (n_users, P, C, custom)
     else:
         n_users, P = args.users or 32, args.prefix or 2048
-        p_lens, s_lens, c_lens = [P] * n_users, [64] * n_users, [512] * n_users
-        workload_name = WORKLOAD if (n_users, P) == (32, 2048) else "config2 model; %d users x (prefix %d cached, 64 short-term, 512 candidates)" % (n_users, P)
+        C = args.candidates or 512
+        p_lens, s_lens, c_lens = [P] * n_users, [64] * n_users, [C] * n_users
+        workload_name = WORKLOAD if (n_users, P, C, custom) == (32, 2048, 512, "") else \
+            "config2 model; %d users x (prefix %d cached, 64 short-term, %d candidates)%s" % (n_users, P, C, custom)
     # replicas: every rank holds its own users (user-hash placement), no data-path collective
     built = workloads.build(shape, wl.seed + 1000 * rank, p_lens, s_lens, c_lens, n_rotations=8, shuffle_pages=args.workload == 3,
                             first_user=rank * n_users, device="cuda:%d" % local)
