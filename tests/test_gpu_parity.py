@@ -325,3 +325,55 @@ def test_two_model_slots_share_one_pool():
     assert report["background_preinfer_calls"] >= 1
     om = oracle_model(shape, w)
     assert max_abs_err(scores, batch, oracle_scores(om, batch)) <= TOL_BF16
+
+
+# ---------------------------------------------------------------- other widths, edge shapes
+@pytest.mark.parametrize("d,heads,ff,layers", [(128, 2, 512, 3), (384, 6, 1536, 2), (1024, 16, 4096, 2)])
+def test_other_model_widths_match_checker(d, heads, ff, layers):
+    """Widths that take the other tile shapes of the GEMM (N not a multiple of 256; the 256-wide long-K tile) and 2 / 6 / 16 heads."""
+    shape = small_bf16_shape(vocab=3000, layers=layers, d=d, heads=heads, ff=ff)
+    batch = _tiny_batch(shape, 50 + d, [333, 64, 129], [7, 0, 65], [70, 130, 1])
+    w, model, pool, db = _setup(shape, 27, batch)
+    om = oracle_model(shape, w)
+    pool.preinfer(db)
+    scores = pool.rank(db).cpu().numpy()
+    full = model.rank_full(db).cpu().numpy()
+    want = oracle_scores(om, batch)
+    assert max_abs_err(scores, batch, want) <= TOL_BF16
+    assert max_abs_err(full, batch, want) <= TOL_BF16
+    assert model.device_status() == 0
+    pool.close(); model.close()
+
+
+def test_degenerate_batches():
+    """No users; users without candidates; one-token prefixes; one user with many candidates over a short prefix (the
+    key range is split across CTAs and merged, with the candidates' own keys folded into the first split)."""
+    B, rt = _runtime()
+    shape = small_bf16_shape()
+    # n_users = 0 is accepted and does nothing
+    w = synth.make_weights(shape, 28)
+    model = rt.Model(shape, w)
+    n0 = model.launch_count()
+    empty = np.zeros(1, dtype=np.int32)
+    B.relaygr_rank_full(model.ctx, 0, None, empty, None, empty, None, empty, None)
+    assert model.launch_count() == n0
+    model.close()
+    # nobody has candidates: nothing to score, but the call is valid
+    batch = _tiny_batch(shape, 91, [65, 1], [3, 0], [0, 0])
+    w, model, pool, db = _setup(shape, 28, batch)
+    pool.preinfer(db)
+    out = pool.rank(db)
+    assert out.numel() == 0 and model.device_status() == 0
+    pool.close(); model.close()
+    # prefixes of 1 and 64 tokens, and a long candidate list against a 1500-token prefix (few items -> split key ranges)
+    batch = _tiny_batch(shape, 92, [1, 64, 1500], [0, 1, 2], [5, 3, 900])
+    w, model, pool, db = _setup(shape, 28, batch)
+    om = oracle_model(shape, w)
+    pool.preinfer(db)
+    scores = pool.rank(db).cpu().numpy()
+    full = model.rank_full(db).cpu().numpy()
+    want = oracle_scores(om, batch)
+    assert max_abs_err(scores, batch, want) <= TOL_BF16
+    assert max_abs_err(full, batch, want) <= TOL_BF16
+    assert model.device_status() == 0
+    pool.close(); model.close()
