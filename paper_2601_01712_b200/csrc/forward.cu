@@ -282,6 +282,7 @@ int Forward::run_t(const CallDesc &call, float *scores, cudaStream_t stream, std
     constexpr bool kTensor = sizeof(T) == 2;
     int *d_status = reinterpret_cast<int *>(ws + lay.status);
     CUtensorMap tm_a, tm_att, tm_hid, tm_q, tm_k, tm_v, tm_pool;
+    GemmOutMaps om_qkv{}, om_hid{}, om_x{};
     if (kTensor) {
         int trc = make_tmap_2d_bf16(&tm_a, a, (uint64_t)R, (uint64_t)d, (uint64_t)d, 128, 64);
         trc |= make_tmap_2d_bf16(&tm_att, att, (uint64_t)R, (uint64_t)d, (uint64_t)d, 128, 64);
@@ -293,12 +294,21 @@ int Forward::run_t(const CallDesc &call, float *scores, cudaStream_t stream, std
             trc |= make_tmap_2d_bf16(&tm_pool, call.pool_slab, (uint64_t)call.pool_pages * L * 2 * 64, (uint64_t)d, (uint64_t)d, 64, 64);
         else
             tm_pool = tm_k;
+        // where the GEMM epilogues store (32-row boxes)
+        trc |= make_tmap_2d_bf16(&om_qkv.o[0], q, (uint64_t)R, (uint64_t)d, (uint64_t)d, 32, 64);
+        trc |= make_tmap_2d_bf16(&om_qkv.o[1], kl, (uint64_t)R, (uint64_t)d, (uint64_t)d, 32, 64);
+        trc |= make_tmap_2d_bf16(&om_qkv.o[2], vl, (uint64_t)R, (uint64_t)d, (uint64_t)d, 32, 64);
+        trc |= make_tmap_2d_bf16(&om_hid.o[0], hid, (uint64_t)R, (uint64_t)F, (uint64_t)F, 32, 64);
+        trc |= make_tmap_2d_f32(&om_x.o[0], x, (uint64_t)R, (uint64_t)d, (uint64_t)d, 32, 32);
+        om_hid.o[1] = om_hid.o[2] = om_hid.o[0];
+        om_x.o[1] = om_x.o[2] = om_x.o[0];
         if (trc != 0) { err = "tensor-map encoding of the activations failed"; return RELAYGR_E_CUDA; }
     }
-    auto gemm = [&](const T *A, const CUtensorMap &tmA, const T *W, const CUtensorMap *tmW, int N, int K, const Epilogue &ep) {
+    auto gemm = [&](const T *A, const CUtensorMap &tmA, const T *W, const CUtensorMap *tmW, const GemmOutMaps &om, int N, int K,
+                    const Epilogue &ep) {
         cudaEvent_t pe = prof_begin(stream);
         cudaError_t r;
-        if constexpr (kTensor) r = launch_gemm_tc(tmA, *tmW, R, N, K, ep, d_status, stream, &launches);
+        if constexpr (kTensor) r = launch_gemm_tc(tmA, *tmW, om, R, N, K, ep, d_status, stream, &launches);
         else r = launch_gemm_simt<T>(A, W, R, N, K, ep, stream, &launches);
         prof_end(KC_GEMM, pe, stream);
         return r;
@@ -338,7 +348,7 @@ int Forward::run_t(const CallDesc &call, float *scores, cudaStream_t stream, std
         if (preinfer) ep.paged = paged;
         const T *Wqkv = (const T *)w.w_qkv + ((size_t)l * 3 * d + ep.col0) * d;
         lm = kTensor ? &wmaps[(size_t)l] : nullptr;
-        e = gemm(a, tm_a, Wqkv, lm ? (kv_only ? &lm->kv : &lm->qkv) : nullptr, 3 * d - ep.col0, d, ep);
+        e = gemm(a, tm_a, Wqkv, lm ? (kv_only ? &lm->kv : &lm->qkv) : nullptr, om_qkv, 3 * d - ep.col0, d, ep);
         if (!ck("QKV projection")) return RELAYGR_E_CUDA;
         if (kv_only) break;
 
@@ -356,7 +366,7 @@ int Forward::run_t(const CallDesc &call, float *scores, cudaStream_t stream, std
 
         Epilogue eo{};
         eo.mode = EPI_RESID; eo.bias = w.b_o ? w.b_o + (size_t)l * d : nullptr; eo.resid = x; eo.out_f32 = x;
-        e = gemm(att, tm_att, (const T *)w.w_o + (size_t)l * d * d, lm ? &lm->wo : nullptr, d, d, eo);
+        e = gemm(att, tm_att, (const T *)w.w_o + (size_t)l * d * d, lm ? &lm->wo : nullptr, om_x, d, d, eo);
         if (!ck("output projection")) return RELAYGR_E_CUDA;
 
         e = layernorm(w.ln2_g + (size_t)l * d, w.ln2_b + (size_t)l * d);
@@ -364,12 +374,12 @@ int Forward::run_t(const CallDesc &call, float *scores, cudaStream_t stream, std
 
         Epilogue e1{};
         e1.mode = EPI_STORE; e1.silu = 1; e1.bias = w.b1 ? w.b1 + (size_t)l * F : nullptr; e1.out = hid;
-        e = gemm(a, tm_a, (const T *)w.w1 + (size_t)l * F * d, lm ? &lm->w1 : nullptr, F, d, e1);
+        e = gemm(a, tm_a, (const T *)w.w1 + (size_t)l * F * d, lm ? &lm->w1 : nullptr, om_hid, F, d, e1);
         if (!ck("FFN 1")) return RELAYGR_E_CUDA;
 
         Epilogue e2{};
         e2.mode = EPI_RESID; e2.bias = w.b2 ? w.b2 + (size_t)l * d : nullptr; e2.resid = x; e2.out_f32 = x;
-        e = gemm(hid, tm_hid, (const T *)w.w2 + (size_t)l * d * F, lm ? &lm->w2 : nullptr, d, F, e2);
+        e = gemm(hid, tm_hid, (const T *)w.w2 + (size_t)l * d * F, lm ? &lm->w2 : nullptr, om_x, d, F, e2);
         if (!ck("FFN 2")) return RELAYGR_E_CUDA;
     }
 

@@ -1,18 +1,20 @@
 // bf16 GEMM on the 5th-generation tensor cores: C[m, n] = sum_k A[m, k] W[n, k] with fp32
 // accumulators in TMEM.  The K extents of this model are short (d_model or d_ff), so a tile's
-// mainloop is a handful of MMAs and the epilogue - reading 128 x 128 accumulators back and
+// mainloop is a handful of MMAs and the epilogue - reading 128 x BN accumulators back and
 // moving them to global memory - is the longer half.  The kernel is therefore persistent
-// (one CTA per SM walks a list of 128 x 128 output tiles) with two accumulators in TMEM, so
+// (one CTA per SM walks a list of 128 x BN output tiles) with two accumulators in TMEM, so
 // that the epilogue of one tile runs under the TMA loads and MMAs of the next, and the
-// epilogue goes through shared memory so that every global access is a full row segment.
+// epilogue hands its output to the TMA unit: a warp stages 32 rows x 128 bytes in shared
+// memory (128-byte swizzle, conflict-free) and one lane issues a bulk tensor store - or, for
+// the residual stream, a bulk fp32 add-reduction (x += tile, performed in L2: the residual
+// never travels to the SM).  Only K/V rows that go straight into a user's pages are written
+// with plain stores (their destination is a page-table walk per row).
 //
 // Warp roles (320 threads): warp 0 = TMA producer (128 x 64 tiles of A and W, 128-byte
-// swizzle, 4-stage ring), warp 1 = TMEM owner + MMA issuer (tcgen05.mma M128 N128 K16),
+// swizzle, 3-4-stage ring), warp 1 = TMEM owner + MMA issuer (tcgen05.mma M128 N = BN K16),
 // warps 2-9 = epilogue: warp w reads TMEM lanes 32 (w % 4) .. +31 (its hardware quadrant),
-// columns 64 ((w - 2) / 4) .. +63 in two chunks of 32, applies bias / SiLU in the
-// row-per-thread layout tcgen05.ld delivers, transposes the chunk through a private
-// shared-memory patch and then reads / writes global memory with 8 (fp32) or 4 (bf16)
-// lanes per row.
+// columns (BN / 2) ((w - 2) / 4) .. + BN / 2 - 1, 64 at a time, applies bias / SiLU in the
+// row-per-thread layout tcgen05.ld delivers and stages the result for the store.
 #include "kernels.cuh"
 #include "tc_common.cuh"
 
@@ -24,17 +26,21 @@ constexpr int BM = 128, BK = 64, kMaxStages = 4;
 constexpr int kEpiWarps = 8;
 constexpr int kThreads = 32 * (2 + kEpiWarps);
 constexpr int kABytes = BM * BK * 2;
-constexpr int kPatchPitchF32 = 36;                                  // floats per staged row (32 + 4 pad): conflict-free float4 access
-constexpr int kPatchBytes = 32 * kPatchPitchF32 * 4;                // 4608 B per warp
+constexpr int kPatchBytes = 32 * 128;                                // one staged store: 32 rows x 128 bytes
+constexpr int kPatches = 2;                                          // per warp: one is filled while the TMA unit reads the other
 
 // Tile width BN: 128, or 256 for long mainloops (gemm_tile_n).  The stage ring is as deep as shared memory allows.
 template <int BN> struct Cfg {
     static constexpr int kBBytes = BN * BK * 2;
     static constexpr int kStage = kABytes + kBBytes;
     static constexpr int kStages = BN == 256 ? 3 : 4;
-    static constexpr int kSmemBytes = kStages * kStage + kEpiWarps * kPatchBytes + kEpiWarps * 32 * 8 /*row offsets*/ + 256 /*barriers*/ +
-                                      1024 /*alignment slack*/;
+    static constexpr int kOffPatch = kStages * kStage;                                    // 1024-byte aligned: stages are
+    static constexpr int kOffBias = kOffPatch + kEpiWarps * kPatches * kPatchBytes;       // per warp BN / 2 floats
+    static constexpr int kOffRowOff = kOffBias + kEpiWarps * (BN / 2) * 4;                // per warp 32 x int64
+    static constexpr int kOffBars = kOffRowOff + kEpiWarps * 32 * 8;
+    static constexpr int kSmemBytes = kOffBars + 256 /*barriers*/ + 1024 /*alignment slack*/;
     static constexpr uint32_t kTmemCols = 2 * BN;
+    static_assert(kSmemBytes <= 227 * 1024, "shared memory budget");
 };
 
 struct GemmBars {
@@ -43,103 +49,35 @@ struct GemmBars {
     uint32_t tmem_slot;
     int abort_flag;
 };
+static_assert(sizeof(GemmBars) <= 256, "barrier block");
 
-// One 32-row x 32-column chunk of the accumulator tile, held one row per lane in v[32].
-// m_base = first row of the warp's quadrant, n = first global output column of the chunk.
-__device__ __forceinline__ void epilogue_chunk(const Epilogue &e, int64_t m_base, int64_t M, int n, int N, float (&v)[32], int lane,
-                                               float *patch, const int64_t *rowoff)
+// 16-byte chunk j of row r of a staged patch (rows of 128 bytes, chunk index XORed with r % 8: the 128-byte swizzle of
+// the output tensor maps, and conflict-free for a warp that writes one row per lane)
+__device__ __forceinline__ uint4 *patch_chunk(uint8_t *patch, int r, int j)
 {
-    if (e.bias) {
-#pragma unroll
-        for (int i = 0; i < 32; i += 4) {
-            const float4 b = *reinterpret_cast<const float4 *>(e.bias + n + i);
-            v[i] += b.x; v[i + 1] += b.y; v[i + 2] += b.z; v[i + 3] += b.w;
-        }
-    }
-    if (e.mode == EPI_RESID) {
-        // stage fp32, then 8 lanes per row: x[m, n .. n+31] += chunk
-        float4 *prow = reinterpret_cast<float4 *>(patch + lane * kPatchPitchF32);
-#pragma unroll
-        for (int i = 0; i < 8; ++i) prow[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
-        __syncwarp();
-        const int rr = lane >> 3, c4 = (lane & 7) * 4;
-        float4 x[8];
-#pragma unroll
-        for (int it = 0; it < 8; ++it) {
-            const int64_t m = m_base + it * 4 + rr;
-            x[it] = m < M ? *reinterpret_cast<const float4 *>(e.resid + m * N + n + c4) : make_float4(0.f, 0.f, 0.f, 0.f);
-        }
-#pragma unroll
-        for (int it = 0; it < 8; ++it) {
-            const int r = it * 4 + rr;
-            const int64_t m = m_base + r;
-            const float4 t = *reinterpret_cast<const float4 *>(patch + r * kPatchPitchF32 + c4);
-            if (m < M) *reinterpret_cast<float4 *>(e.out_f32 + m * N + n + c4) = make_float4(x[it].x + t.x, x[it].y + t.y, x[it].z + t.z, x[it].w + t.w);
-        }
-        __syncwarp();
-        return;
-    }
-    if (e.mode == EPI_STORE && e.silu) {
-        // SiLU(z) = z sigmoid(z) = h + h tanh(h), h = z / 2: one MUFU op per element (tanh.approx, relative error 2^-11,
-        // below the bf16 rounding of the result that follows)
-#pragma unroll
-        for (int i = 0; i < 32; ++i) {
-            const float h = 0.5f * v[i];
-            float t;
-            asm("tanh.approx.f32 %0, %1;" : "=f"(t) : "f"(h));
-            v[i] = fmaf(h, t, h);
-        }
-    }
-    // bf16 outputs: stage 64-byte rows (pitch 80 bytes), then 4 lanes per row write 16 bytes each
-    constexpr int kPitchB = 80;
-    uint8_t *pb = reinterpret_cast<uint8_t *>(patch);
-    uint4 *prow = reinterpret_cast<uint4 *>(pb + lane * kPitchB);
-#pragma unroll
-    for (int i = 0; i < 4; ++i)
-        prow[i] = make_uint4(tc::pack_bf16(v[8 * i], v[8 * i + 1]), tc::pack_bf16(v[8 * i + 2], v[8 * i + 3]),
-                             tc::pack_bf16(v[8 * i + 4], v[8 * i + 5]), tc::pack_bf16(v[8 * i + 6], v[8 * i + 7]));
-    __syncwarp();
-    // where the chunk's rows go
-    __nv_bfloat16 *base;          // element (row 0 of the call, column c of this chunk)
-    int64_t pitch;                // elements between rows of the call (unused for the paged scatter)
-    bool paged = false;
-    int which = 0, c = n;
-    if (e.mode == EPI_STORE) {
-        base = reinterpret_cast<__nv_bfloat16 *>(e.out) + n; pitch = N;
-    } else {
-        const int col = e.col0 + n, d = e.d_model;
-        which = col / d; c = col - which * d;
-        pitch = d;
-        if (which == 0) base = reinterpret_cast<__nv_bfloat16 *>(e.q) + c;
-        else if (!e.paged.slab) base = reinterpret_cast<__nv_bfloat16 *>(which == 1 ? e.k_lin : e.v_lin) + c;
-        else { paged = true; base = reinterpret_cast<__nv_bfloat16 *>(e.paged.slab) + (size_t)(which - 1) * 64 * d + c; }
-    }
-    const int rr = lane >> 2, c8 = (lane & 3) * 8;
-#pragma unroll
-    for (int it = 0; it < 4; ++it) {
-        const int r = it * 8 + rr;
-        const int64_t m = m_base + r;
-        if (m < M) {
-            const uint4 t = *reinterpret_cast<const uint4 *>(pb + r * kPitchB + (lane & 3) * 16);
-            __nv_bfloat16 *dst = paged ? base + rowoff[r] + c8 : base + m * pitch + c8;
-            *reinterpret_cast<uint4 *>(dst) = t;
-        }
-    }
-    __syncwarp();
+    return reinterpret_cast<uint4 *>(patch + r * 128 + ((j ^ (r & 7)) << 4));
+}
+
+// SiLU(z) = z sigmoid(z) = h + h tanh(h), h = z / 2: one MUFU op per element (tanh.approx, relative error 2^-11, below
+// the bf16 rounding of the result that follows)
+__device__ __forceinline__ float silu(float z)
+{
+    const float h = 0.5f * z;
+    float t;
+    asm("tanh.approx.f32 %0, %1;" : "=f"(t) : "f"(h));
+    return fmaf(h, t, h);
 }
 
 template <int BN>
 __global__ void __launch_bounds__(kThreads, 1)
-gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, int64_t M, int N, int K,
-               Epilogue epi, int *err)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const __grid_constant__ GemmOutMaps om,
+               int64_t M, int N, int K, Epilogue epi, int *err)
 {
     constexpr int STAGES = Cfg<BN>::kStages, kStage = Cfg<BN>::kStage;
     constexpr uint32_t kTmemCols = Cfg<BN>::kTmemCols;
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    float *patches = reinterpret_cast<float *>(smem + STAGES * kStage);
-    int64_t *rowoffs = reinterpret_cast<int64_t *>(smem + STAGES * kStage + kEpiWarps * kPatchBytes);
-    GemmBars *bars = reinterpret_cast<GemmBars *>(smem + STAGES * kStage + kEpiWarps * kPatchBytes + kEpiWarps * 32 * 8);
+    GemmBars *bars = reinterpret_cast<GemmBars *>(smem + Cfg<BN>::kOffBars);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int kblocks = K / BK;
@@ -222,20 +160,45 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         const int quad = warp & 3;                          // TMEM lanes this warp may touch: 32*quad .. 32*quad+31
         const int half = ew >> 2;                           // columns (BN/2)*half .. +BN/2-1 of the tile, 64 at a time
         constexpr int kColsPerWarp = BN / 2;
-        float *patch = patches + ew * (kPatchBytes / 4);
-        int64_t *rowoff = rowoffs + ew * 32;
+        uint8_t *patches = smem + Cfg<BN>::kOffPatch + ew * (kPatches * kPatchBytes);
+        float *bias_s = reinterpret_cast<float *>(smem + Cfg<BN>::kOffBias) + ew * kColsPerWarp;
+        int64_t *rowoff = reinterpret_cast<int64_t *>(smem + Cfg<BN>::kOffRowOff) + ew * 32;
         const bool scatter = epi.mode == EPI_QKV && epi.paged.slab != nullptr;
+        uint32_t pp = 0;                                    // the patch the next staged store fills
+        // the store that filled this patch last has read it (the one in flight may still read the other patch)
+        auto patch_acquire = [&]() -> uint8_t * {
+            if (lane == 0) tc::bulk_wait_read<kPatches - 1>();
+            __syncwarp();
+            return patches + pp * kPatchBytes;
+        };
+        // every lane has written its row: hand the patch to the TMA unit
+        auto patch_submit = [&](const CUtensorMap *map, const uint8_t *patch, int x, int y, bool add) {
+            tc::fence_proxy_async();
+            __syncwarp();
+            if (lane == 0) {
+                if (add) tc::tma_reduce_add_2d(map, patch, x, y);
+                else tc::tma_store_2d(map, patch, x, y);
+                tc::bulk_commit();
+            }
+            pp ^= 1;
+        };
         uint32_t ti = 0;
         bool ok = true;
         for (int64_t t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++ti) {
             const int64_t m0 = (t / n_tiles_n) * BM;
-            const int n0 = (int)(t % n_tiles_n) * BN;
+            const int n_w = (int)(t % n_tiles_n) * BN + half * kColsPerWarp;      // first column of this warp's part
             const uint32_t as = ti & 1;
             const int64_t m_base = m0 + quad * 32;
             const int64_t m = m_base + lane;
-            // K / V rows of a pre-infer call go straight into the user's pages: offset of (page, K, slot) per row
+            // before the accumulator is ready: this warp's slice of the bias, and for K / V rows of a pre-infer call
+            // (they go straight into the user's pages) the offset of (page, K, slot) per row
+            if (epi.bias) {
+#pragma unroll
+                for (int c = 0; c < kColsPerWarp; c += 32) bias_s[c + lane] = epi.bias[n_w + c + lane];
+            }
             int last_slot = -1, page = 0;
-            if (scatter && epi.col0 + n0 + half * kColsPerWarp + kColsPerWarp - 1 >= epi.d_model) {
+            const bool paged_tile = scatter && epi.col0 + n_w + kColsPerWarp - 1 >= epi.d_model;
+            if (paged_tile) {
                 int64_t off = 0;
                 if (m < M) {
                     const int u = find_user(epi.row_off, epi.n_users, (int)m);
@@ -245,8 +208,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     if (tt == epi.seqs[u].n_q - 1) last_slot = tt & 63;
                 }
                 rowoff[lane] = off;
-                __syncwarp();
             }
+            __syncwarp();
             ok = __all_sync(0xffffffffu, tc::mbar_wait(&bars->acc_full[as], (ti >> 1) & 1, err));
             if (!ok) break;
             tc::tc_fence_after();
@@ -262,26 +225,98 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     __syncwarp();
                     if (lane == 0) tc::mbar_arrive(&bars->acc_empty[as]);      // this warp's part of the accumulator is in registers
                 }
-                float v[32];
+                if (m_base >= M) continue;                                       // the whole row group lies past the last row
+                const int n = n_w + pass * 64;                                   // first output column of these 64
+                if (epi.bias) {
+                    const float4 *b4 = reinterpret_cast<const float4 *>(bias_s + pass * 64);
 #pragma unroll
-                for (int cc = 0; cc < 2; ++cc) {
+                    for (int i = 0; i < 8; ++i) {
+                        const float4 b = b4[i], c = b4[8 + i];
+                        r0[4 * i] = __float_as_uint(__uint_as_float(r0[4 * i]) + b.x);
+                        r0[4 * i + 1] = __float_as_uint(__uint_as_float(r0[4 * i + 1]) + b.y);
+                        r0[4 * i + 2] = __float_as_uint(__uint_as_float(r0[4 * i + 2]) + b.z);
+                        r0[4 * i + 3] = __float_as_uint(__uint_as_float(r0[4 * i + 3]) + b.w);
+                        r1[4 * i] = __float_as_uint(__uint_as_float(r1[4 * i]) + c.x);
+                        r1[4 * i + 1] = __float_as_uint(__uint_as_float(r1[4 * i + 1]) + c.y);
+                        r1[4 * i + 2] = __float_as_uint(__uint_as_float(r1[4 * i + 2]) + c.z);
+                        r1[4 * i + 3] = __float_as_uint(__uint_as_float(r1[4 * i + 3]) + c.w);
+                    }
+                }
+                if (epi.mode == EPI_RESID) {
+                    // x[m, n .. n+63] += tile, as two fp32 patches of 32 columns
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(cc == 0 ? r0[i] : r1[i]);
-                    const int n = n0 + half * kColsPerWarp + pass * 64 + cc * 32;
-                    epilogue_chunk(epi, m_base, M, n, N, v, lane, patch, rowoff);
-                    if (last_slot >= 0 && last_slot < 63 && epi.col0 + n >= epi.d_model) {
-                        // last prefix row of a user: clear the unused slots of its last page (they are masked, but must hold finite values)
-                        const int col = epi.col0 + n, which = col / epi.d_model, c = col - which * epi.d_model;
-                        __nv_bfloat16 *slab = reinterpret_cast<__nv_bfloat16 *>(epi.paged.slab);
-                        const uint4 z = make_uint4(0, 0, 0, 0);
-                        for (int s = last_slot + 1; s < 64; ++s) {
-                            uint4 *zp = reinterpret_cast<uint4 *>(slab + page_elem_offset(epi.paged, page, which - 1, s) + c);
-                            zp[0] = z; zp[1] = z; zp[2] = z; zp[3] = z;
-                        }
+                    for (int cc = 0; cc < 2; ++cc) {
+                        uint8_t *patch = patch_acquire();
+#pragma unroll
+                        for (int j = 0; j < 8; ++j)
+                            *patch_chunk(patch, lane, j) = cc == 0 ? make_uint4(r0[4 * j], r0[4 * j + 1], r0[4 * j + 2], r0[4 * j + 3])
+                                                                   : make_uint4(r1[4 * j], r1[4 * j + 1], r1[4 * j + 2], r1[4 * j + 3]);
+                        patch_submit(&om.o[0], patch, n + cc * 32, (int)m_base, true);
+                    }
+                    continue;
+                }
+                if (epi.mode == EPI_STORE && epi.silu) {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) {
+                        r0[i] = __float_as_uint(silu(__uint_as_float(r0[i])));
+                        r1[i] = __float_as_uint(silu(__uint_as_float(r1[i])));
+                    }
+                }
+                // bf16 outputs: 64 columns = one 128-byte row per lane
+                int which = 0, c = n;                                            // destination tensor and its column
+                if (epi.mode == EPI_QKV) {
+                    const int col = epi.col0 + n;
+                    which = col / epi.d_model; c = col - which * epi.d_model;
+                }
+                const bool paged = paged_tile && which > 0;
+                uint8_t *patch;
+                if (paged) {
+                    if (lane == 0) tc::bulk_wait_read<0>();                      // both patches idle: this path reads its own staging
+                    __syncwarp();
+                    patch = patches;
+                } else {
+                    patch = patch_acquire();
+                }
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    *patch_chunk(patch, lane, j) =
+                        make_uint4(tc::pack_bf16(__uint_as_float(r0[8 * j]), __uint_as_float(r0[8 * j + 1])),
+                                   tc::pack_bf16(__uint_as_float(r0[8 * j + 2]), __uint_as_float(r0[8 * j + 3])),
+                                   tc::pack_bf16(__uint_as_float(r0[8 * j + 4]), __uint_as_float(r0[8 * j + 5])),
+                                   tc::pack_bf16(__uint_as_float(r0[8 * j + 6]), __uint_as_float(r0[8 * j + 7])));
+                    *patch_chunk(patch, lane, 4 + j) =
+                        make_uint4(tc::pack_bf16(__uint_as_float(r1[8 * j]), __uint_as_float(r1[8 * j + 1])),
+                                   tc::pack_bf16(__uint_as_float(r1[8 * j + 2]), __uint_as_float(r1[8 * j + 3])),
+                                   tc::pack_bf16(__uint_as_float(r1[8 * j + 4]), __uint_as_float(r1[8 * j + 5])),
+                                   tc::pack_bf16(__uint_as_float(r1[8 * j + 6]), __uint_as_float(r1[8 * j + 7])));
+                }
+                if (!paged) {
+                    patch_submit(&om.o[which], patch, c, (int)m_base, false);
+                    continue;
+                }
+                // K / V rows into pages: 8 lanes per row copy its 128 bytes to (page, K | V, slot)
+                __syncwarp();
+                __nv_bfloat16 *kv = reinterpret_cast<__nv_bfloat16 *>(epi.paged.slab) + (size_t)(which - 1) * 64 * epi.d_model + c;
+                const int rr = lane >> 3, cj = lane & 7;
+#pragma unroll
+                for (int it = 0; it < 8; ++it) {
+                    const int r = it * 4 + rr;
+                    if (m_base + r < M) *reinterpret_cast<uint4 *>(kv + rowoff[r] + cj * 8) = *patch_chunk(patch, r, cj);
+                }
+                __syncwarp();
+                if (last_slot >= 0 && last_slot < 63) {
+                    // last prefix row of a user: clear the unused slots of its last page (they are masked, but must hold finite values)
+                    __nv_bfloat16 *slab = reinterpret_cast<__nv_bfloat16 *>(epi.paged.slab);
+                    const uint4 z = make_uint4(0, 0, 0, 0);
+                    for (int s = last_slot + 1; s < 64; ++s) {
+                        uint4 *zp = reinterpret_cast<uint4 *>(slab + page_elem_offset(epi.paged, page, which - 1, s) + c);
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) zp[j] = z;
                     }
                 }
             }
         }
+        if (lane == 0) tc::bulk_wait<0>();                  // this warp's stores have been performed
     }
     tc::tc_fence_before();
     __syncthreads();
@@ -291,8 +326,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 }  // namespace
 
 template <int BN>
-static cudaError_t launch_bn(const CUtensorMap &tmA, const CUtensorMap &tmB, int64_t M, int N, int K, const Epilogue &epi, int *err,
-                             cudaStream_t stream)
+static cudaError_t launch_bn(const CUtensorMap &tmA, const CUtensorMap &tmB, const GemmOutMaps &om, int64_t M, int N, int K,
+                             const Epilogue &epi, int *err, cudaStream_t stream)
 {
     static int n_sms = 0;
     if (n_sms == 0) {
@@ -304,15 +339,15 @@ static cudaError_t launch_bn(const CUtensorMap &tmA, const CUtensorMap &tmB, int
     }
     const int64_t tiles = ((M + BM - 1) / BM) * (N / BN);
     const unsigned grid = (unsigned)(tiles < n_sms ? tiles : n_sms);
-    return launch_dependent(gemm_tc_kernel<BN>, dim3(grid), dim3(kThreads), (size_t)Cfg<BN>::kSmemBytes, stream, tmA, tmB, M, N, K, epi, err);
+    return launch_dependent(gemm_tc_kernel<BN>, dim3(grid), dim3(kThreads), (size_t)Cfg<BN>::kSmemBytes, stream, tmA, tmB, om, M, N, K, epi, err);
 }
 
-cudaError_t launch_gemm_tc(const CUtensorMap &tmA, const CUtensorMap &tmB, int64_t M, int N, int K, const Epilogue &epi,
-                           int *err, cudaStream_t stream, int64_t *launches)
+cudaError_t launch_gemm_tc(const CUtensorMap &tmA, const CUtensorMap &tmB, const GemmOutMaps &om, int64_t M, int N, int K,
+                           const Epilogue &epi, int *err, cudaStream_t stream, int64_t *launches)
 {
     if (M == 0 || N == 0) return cudaSuccess;
     *launches += 1;
-    return gemm_tile_n(N, K) == 256 ? launch_bn<256>(tmA, tmB, M, N, K, epi, err, stream) : launch_bn<128>(tmA, tmB, M, N, K, epi, err, stream);
+    return gemm_tile_n(N, K) == 256 ? launch_bn<256>(tmA, tmB, om, M, N, K, epi, err, stream) : launch_bn<128>(tmA, tmB, om, M, N, K, epi, err, stream);
 }
 
 }  // namespace relaygr

@@ -62,16 +62,21 @@ cudaError_t launch_attention_simt(const T *q, const T *k_lin, const T *v_lin, Pa
 
 // ---- tensor-core kernels (the bf16 model) -------------------------------------------------------------
 
-// Output tile width of the tensor-core GEMM for [*, K] x [N, K]^T (N % 128 == 0): 256 pays only when the mainloop is
-// long (K >= 1024: twice the MMA work per pipeline hand-shake, A read once per 256 columns); with the short K of the
-// other projections the longer epilogue of a wide tile costs more than that gains (measured).
-inline int gemm_tile_n(int N, int K) { return (N % 256 == 0 && K >= 1024) ? 256 : 128; }
+// Output tile width of the tensor-core GEMM for [*, K] x [N, K]^T (N % 128 == 0).  A 256-wide tile does twice the MMA
+// work per pipeline hand-shake and per issued instruction, and reads A once per 256 columns; it pays from K = 512 on
+// (measured).  At K = 256 a tile is eight instructions either way and the finer 128-wide tiles balance better.
+inline int gemm_tile_n(int N, int K) { return (N % 256 == 0 && K >= 512) ? 256 : 128; }
+
+// Where a GEMM's epilogue stores: tensor maps with a 32-row box of 128 bytes and the 128-byte swizzle.
+// EPI_STORE: o[0] = out [M, N] bf16.  EPI_RESID: o[0] = the fp32 residual stream [M, N] (tile added in place).
+// EPI_QKV: o[0] = q, o[1] = k_lin, o[2] = v_lin, each [M, d] bf16 (o[1], o[2] are not used when K / V go to pages).
+struct GemmOutMaps { CUtensorMap o[3]; };
 
 // C[m, n] = sum_k A[m, k] W[n, k] on tcgen05; tmA covers A [M, K] with a 128-row box, tmB covers W [N, K]
 // with a box of gemm_tile_n(N, K) rows, both 64 columns wide with the 128-byte swizzle.  N % 128 == 0, K % 64 == 0.
 // err is a device status word: kernels record a code there instead of hanging or trapping.
-cudaError_t launch_gemm_tc(const CUtensorMap &tmA, const CUtensorMap &tmB, int64_t M, int N, int K, const Epilogue &epi,
-                           int *err, cudaStream_t stream, int64_t *launches);
+cudaError_t launch_gemm_tc(const CUtensorMap &tmA, const CUtensorMap &tmB, const GemmOutMaps &om, int64_t M, int N, int K,
+                           const Epilogue &epi, int *err, cudaStream_t stream, int64_t *launches);
 
 // Flash-style attention on tcgen05 (d_head = 64) over the work items, then the merge of split items.
 // tmQ: [rows, d] box 128 x 64; tmK / tmV: the call's transient K / V rows, box 64 x 64; tmPool: the pool

@@ -20,20 +20,33 @@ PFN_cuTensorMapEncodeTiled_v12000 get_encode()
 }
 }  // namespace
 
-int make_tmap_2d_bf16(CUtensorMap *out, const void *base, uint64_t rows, uint64_t cols, uint64_t pitch_elems,
-                      uint32_t box_rows, uint32_t box_cols)
+namespace {
+int encode_2d(CUtensorMap *out, CUtensorMapDataType type, uint32_t elem_bytes, const void *base, uint64_t rows, uint64_t cols,
+              uint64_t pitch_elems, uint32_t box_rows, uint32_t box_cols)
 {
     PFN_cuTensorMapEncodeTiled_v12000 enc = get_encode();
     if (!enc) return -1;
-    if ((reinterpret_cast<uintptr_t>(base) & 15) != 0 || (pitch_elems * 2) % 16 != 0 || box_cols * 2 != 128) return -2;
+    if ((reinterpret_cast<uintptr_t>(base) & 15) != 0 || (pitch_elems * elem_bytes) % 16 != 0 || box_cols * elem_bytes != 128) return -2;
     const cuuint64_t dims[2] = {cols, rows};
-    const cuuint64_t strides[1] = {pitch_elems * 2};
+    const cuuint64_t strides[1] = {pitch_elems * elem_bytes};
     const cuuint32_t box[2] = {box_cols, box_rows};
     const cuuint32_t estr[2] = {1, 1};
-    const CUresult r = enc(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
-                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    const CUresult r = enc(out, type, 2, const_cast<void *>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                           CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? 0 : -3;
+}
+}  // namespace
+
+int make_tmap_2d_bf16(CUtensorMap *out, const void *base, uint64_t rows, uint64_t cols, uint64_t pitch_elems,
+                      uint32_t box_rows, uint32_t box_cols)
+{
+    return encode_2d(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, rows, cols, pitch_elems, box_rows, box_cols);
+}
+
+int make_tmap_2d_f32(CUtensorMap *out, const void *base, uint64_t rows, uint64_t cols, uint64_t pitch_elems,
+                     uint32_t box_rows, uint32_t box_cols)
+{
+    return encode_2d(out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, base, rows, cols, pitch_elems, box_rows, box_cols);
 }
 
 }  // namespace relaygr
