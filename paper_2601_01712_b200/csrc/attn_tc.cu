@@ -439,11 +439,11 @@ cudaError_t launch_attention_tc(const CUtensorMap &tmQ, const CUtensorMap &tmK, 
         attr_set = true;
     }
     *launches += 1;
-    cudaError_t e = launch_dependent(attention_tc_kernel, dim3(n_items), dim3(192), (size_t)kSmemBytes, stream, tmQ, tmK, tmV, tmPool, items,
+    cudaError_t e = launch_dependent(attention_tc_kernel, dim3(n_items), dim3(192), (size_t)kSmemBytes, stream, 1, tmQ, tmK, tmV, tmPool, items,
                                      seqs, pt, n_layers, layer, d_model, q, k_lin, v_lin, out, partial, err);
     if (e != cudaSuccess || n_merges == 0) return e;
     *launches += 1;
-    return launch_dependent(attention_merge_kernel, dim3(n_merges, kQTile / 8), dim3(256), 0, stream, merges, seqs, partial, d_model, out);
+    return launch_dependent(attention_merge_kernel, dim3(n_merges, kQTile / 8), dim3(256), 0, stream, 1, merges, seqs, partial, d_model, out);
 }
 
 }  // namespace relaygr

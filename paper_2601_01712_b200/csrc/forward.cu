@@ -77,11 +77,11 @@ int Forward::init_device(int dev, std::string &err)
         wmaps.resize((size_t)cfg.n_layers);
         for (int l = 0; l < cfg.n_layers; ++l) {
             const __nv_bfloat16 *wq = (const __nv_bfloat16 *)w.w_qkv + (size_t)l * 3 * d * d;
-            int rc = make_tmap_2d_bf16(&wmaps[(size_t)l].qkv, wq, 3 * d, d, d, (uint32_t)gemm_tile_n((int)(3 * d), (int)d), 64);
-            rc |= make_tmap_2d_bf16(&wmaps[(size_t)l].kv, wq + d * d, 2 * d, d, d, (uint32_t)gemm_tile_n((int)(2 * d), (int)d), 64);
-            rc |= make_tmap_2d_bf16(&wmaps[(size_t)l].wo, (const __nv_bfloat16 *)w.w_o + (size_t)l * d * d, d, d, d, (uint32_t)gemm_tile_n((int)d, (int)d), 64);
-            rc |= make_tmap_2d_bf16(&wmaps[(size_t)l].w1, (const __nv_bfloat16 *)w.w1 + (size_t)l * F * d, F, d, d, (uint32_t)gemm_tile_n((int)F, (int)d), 64);
-            rc |= make_tmap_2d_bf16(&wmaps[(size_t)l].w2, (const __nv_bfloat16 *)w.w2 + (size_t)l * d * F, d, F, F, (uint32_t)gemm_tile_n((int)d, (int)F), 64);
+            int rc = make_tmap_2d_bf16(&wmaps[(size_t)l].qkv, wq, 3 * d, d, d, (uint32_t)kGemmWeightBoxRows, 64);
+            rc |= make_tmap_2d_bf16(&wmaps[(size_t)l].kv, wq + d * d, 2 * d, d, d, (uint32_t)kGemmWeightBoxRows, 64);
+            rc |= make_tmap_2d_bf16(&wmaps[(size_t)l].wo, (const __nv_bfloat16 *)w.w_o + (size_t)l * d * d, d, d, d, (uint32_t)kGemmWeightBoxRows, 64);
+            rc |= make_tmap_2d_bf16(&wmaps[(size_t)l].w1, (const __nv_bfloat16 *)w.w1 + (size_t)l * F * d, F, d, d, (uint32_t)kGemmWeightBoxRows, 64);
+            rc |= make_tmap_2d_bf16(&wmaps[(size_t)l].w2, (const __nv_bfloat16 *)w.w2 + (size_t)l * d * F, d, F, F, (uint32_t)kGemmWeightBoxRows, 64);
             if (rc != 0) { err = "tensor-map encoding of the weights failed (pointers must be 16-byte aligned)"; return RELAYGR_E_CUDA; }
         }
     }

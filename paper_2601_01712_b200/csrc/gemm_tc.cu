@@ -22,18 +22,22 @@ namespace relaygr {
 
 namespace {
 
-constexpr int BM = 128, BK = 64, kMaxStages = 4;
+constexpr int BM = 128, BK = 64, kMaxStages = 5;
 constexpr int kEpiWarps = 8;
 constexpr int kThreads = 32 * (2 + kEpiWarps);
 constexpr int kABytes = BM * BK * 2;
 constexpr int kPatchBytes = 32 * 128;                                // one staged store: 32 rows x 128 bytes
-constexpr int kPatches = 2;                                          // per warp: one is filled while the TMA unit reads the other
+constexpr int kPatches = 1;                                          // per warp (a store has read its patch long before the next is packed)
 
-// Tile width BN: 128, or 256 for long mainloops (gemm_tile_n).  The stage ring is as deep as shared memory allows.
-template <int BN> struct Cfg {
-    static constexpr int kBBytes = BN * BK * 2;
+// A tile is 128 x BN per CTA.  CTAS = 1: BN = 128 (or 256), the CTA loads all of A and B.  CTAS = 2: a pair of CTAs works on
+// 256 x 256 with one tcgen05 cta_group::2 MMA stream issued by the even CTA; each CTA loads its 128 rows of A and half
+// (128 rows) of B, so a K block costs each CTA 32 KB of shared-memory writes and 32 KB of operand reads per 512 tensor
+// clocks - the shared-memory bandwidth that a single CTA spends on 128 x 128.  The stage ring is as deep as shared
+// memory allows.
+template <int BN, int CTAS> struct Cfg {
+    static constexpr int kBBytes = (BN / CTAS) * BK * 2;
     static constexpr int kStage = kABytes + kBBytes;
-    static constexpr int kStages = BN == 256 ? 3 : 4;
+    static constexpr int kStages = (CTAS == 1 && BN == 256) ? 3 : 5;
     static constexpr int kOffPatch = kStages * kStage;                                    // 1024-byte aligned: stages are
     static constexpr int kOffBias = kOffPatch + kEpiWarps * kPatches * kPatchBytes;       // per warp BN / 2 floats
     static constexpr int kOffRowOff = kOffBias + kEpiWarps * (BN / 2) * 4;                // per warp 32 x int64
@@ -41,6 +45,7 @@ template <int BN> struct Cfg {
     static constexpr int kSmemBytes = kOffBars + 256 /*barriers*/ + 1024 /*alignment slack*/;
     static constexpr uint32_t kTmemCols = 2 * BN;
     static_assert(kSmemBytes <= 227 * 1024, "shared memory budget");
+    static_assert(CTAS == 1 || BN == 256, "a CTA pair works on 256 x 256");
 };
 
 struct GemmBars {
@@ -68,34 +73,39 @@ __device__ __forceinline__ float silu(float z)
     return fmaf(h, t, h);
 }
 
-template <int BN>
+template <int BN, int CTAS>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const __grid_constant__ GemmOutMaps om,
                int64_t M, int N, int K, Epilogue epi, int *err)
 {
-    constexpr int STAGES = Cfg<BN>::kStages, kStage = Cfg<BN>::kStage;
-    constexpr uint32_t kTmemCols = Cfg<BN>::kTmemCols;
+    using C = Cfg<BN, CTAS>;
+    constexpr int STAGES = C::kStages, kStage = C::kStage;
+    constexpr uint32_t kTmemCols = C::kTmemCols;
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    GemmBars *bars = reinterpret_cast<GemmBars *>(smem + Cfg<BN>::kOffBars);
+    GemmBars *bars = reinterpret_cast<GemmBars *>(smem + C::kOffBars);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int kblocks = K / BK;
     const int n_tiles_n = N / BN;
-    const int64_t n_tiles = ((M + BM - 1) / BM) * n_tiles_n;
+    const int64_t n_tiles = ((M + BM * CTAS - 1) / (BM * CTAS)) * n_tiles_n;       // tiles of the CTA (or the pair)
+    const uint32_t rank = CTAS == 2 ? tc::cluster_ctarank() : 0;                     // this CTA's half of a pair tile
+    const int64_t worker = blockIdx.x / CTAS, n_workers = gridDim.x / CTAS;
+    const bool leader = rank == 0;                                                   // issues the MMAs, owns full / acc_empty
 
     // set-up that touches nothing earlier kernels wrote; it may run while the previous kernel is still finishing
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { tc::mbar_init(&bars->full[s], 1); tc::mbar_init(&bars->empty[s], 1); }
-        for (int s = 0; s < 2; ++s) { tc::mbar_init(&bars->acc_full[s], 1); tc::mbar_init(&bars->acc_empty[s], kEpiWarps); }
+        for (int s = 0; s < 2; ++s) { tc::mbar_init(&bars->acc_full[s], 1); tc::mbar_init(&bars->acc_empty[s], kEpiWarps * CTAS); }
         tc::fence_mbar_init();
         tc::tma_prefetch_desc(&tmA);
         tc::tma_prefetch_desc(&tmB);
     }
     if (warp == 1) {
-        tc::tmem_alloc(&bars->tmem_slot, kTmemCols);
-        tc::tmem_relinquish();
+        if constexpr (CTAS == 2) { tc::tmem_alloc_pair(&bars->tmem_slot, kTmemCols); tc::tmem_relinquish_pair(); }
+        else { tc::tmem_alloc(&bars->tmem_slot, kTmemCols); tc::tmem_relinquish(); }
     }
+    if constexpr (CTAS == 2) tc::cluster_sync();                  // the peer's barriers exist before anything signals them
     grid_launch_dependents();
     grid_dependency_wait();                                       // from here on: data of earlier kernels
     if (threadIdx.x == 0) bars->abort_flag = *reinterpret_cast<volatile int *>(err);
@@ -107,31 +117,40 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
     if (!live) {
     } else if (warp == 0) {
-        // ---------------------------------------------------------------- TMA producer
+        // ---------------------------------------------------------------- TMA producer: this CTA's rows of A and of B
         if (lane == 0) {
             uint32_t it = 0;
             bool ok = true;
-            for (int64_t t = blockIdx.x; t < n_tiles && ok; t += gridDim.x) {
-                const int m0 = (int)(t / n_tiles_n) * BM, n0 = (int)(t % n_tiles_n) * BN;
+            for (int64_t t = worker; t < n_tiles && ok; t += n_workers) {
+                const int m0 = (int)(t / n_tiles_n) * (BM * CTAS) + (int)rank * BM;
+                const int n0 = (int)(t % n_tiles_n) * BN + (int)rank * (BN / CTAS);
                 for (int kb = 0; kb < kblocks; ++kb, ++it) {
                     const int s = it % STAGES;
                     ok = tc::mbar_wait(&bars->empty[s], ((it / STAGES) & 1) ^ 1, err);
                     if (!ok) break;
-                    tc::mbar_expect_tx(&bars->full[s], kStage);
                     uint8_t *a = smem + s * kStage;
-                    tc::tma_load_2d(a, &tmA, kb * BK, m0, &bars->full[s]);
-                    tc::tma_load_2d(a + kABytes, &tmB, kb * BK, n0, &bars->full[s]);
+                    if constexpr (CTAS == 2) {
+                        // both CTAs' bytes are counted on the even CTA's barrier, which expects the sum
+                        if (leader) tc::mbar_expect_tx(&bars->full[s], 2 * kStage);
+                        const uint32_t bar = tc::cluster_addr(&bars->full[s], 0);
+                        tc::tma_load_2d_pair(a, &tmA, kb * BK, m0, bar);
+                        tc::tma_load_2d_pair(a + kABytes, &tmB, kb * BK, n0, bar);
+                    } else {
+                        tc::mbar_expect_tx(&bars->full[s], kStage);
+                        tc::tma_load_2d(a, &tmA, kb * BK, m0, &bars->full[s]);
+                        tc::tma_load_2d(a + kABytes, &tmB, kb * BK, n0, &bars->full[s]);
+                    }
                 }
             }
         }
     } else if (warp == 1) {
         // ---------------------------------------------------------------- MMA issuer (the whole warp walks the loop so that
-        // addresses stay warp-uniform; one elected lane issues the tcgen05 instructions)
-        {
-            constexpr uint32_t idesc = tc::make_idesc(BM, BN, 0, 0);
+        // addresses stay warp-uniform; one elected lane issues the tcgen05 instructions).  In a pair only the even CTA issues.
+        if (leader) {
+            constexpr uint32_t idesc = tc::make_idesc(BM * CTAS, BN, 0, 0);
             uint32_t it = 0, ti = 0;
             bool ok = true;
-            for (int64_t t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++ti) {
+            for (int64_t t = worker; t < n_tiles && ok; t += n_workers, ++ti) {
                 const uint32_t as = ti & 1;
                 ok = tc::mbar_wait(&bars->acc_empty[as], ((ti >> 1) & 1) ^ 1, err);     // the epilogue has drained this accumulator
                 if (!ok) break;
@@ -144,11 +163,21 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     const uint32_t a = tc::smem_u32(smem + s * kStage);
                     const uint64_t adesc = tc::smem_desc_sw128(a), bdesc = tc::smem_desc_sw128(a + kABytes);
                     if (tc::elect_one()) {
+                        // 32 bytes of K per instruction: descriptor start address + 2.  A commit frees the stage (in both
+                        // CTAs of a pair) when these MMAs have read it; the last one also hands the accumulator over.
+                        if constexpr (CTAS == 2) {
 #pragma unroll
-                        for (int k = 0; k < BK / 16; ++k)     // 32 bytes of K per instruction: descriptor start address + 2
-                            tc::mma_ss(tmem_base + as * BN, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0);
-                        tc::mma_commit(&bars->empty[s]);       // frees the stage when these MMAs have read it
-                        if (kb == kblocks - 1) tc::mma_commit(&bars->acc_full[as]);
+                            for (int k = 0; k < BK / 16; ++k)
+                                tc::mma_ss_pair(tmem_base + as * BN, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0);
+                            tc::mma_commit_pair(&bars->empty[s], 3);
+                            if (kb == kblocks - 1) tc::mma_commit_pair(&bars->acc_full[as], 3);
+                        } else {
+#pragma unroll
+                            for (int k = 0; k < BK / 16; ++k)
+                                tc::mma_ss(tmem_base + as * BN, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0);
+                            tc::mma_commit(&bars->empty[s]);
+                            if (kb == kblocks - 1) tc::mma_commit(&bars->acc_full[as]);
+                        }
                     }
                     __syncwarp();
                 }
@@ -160,9 +189,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         const int quad = warp & 3;                          // TMEM lanes this warp may touch: 32*quad .. 32*quad+31
         const int half = ew >> 2;                           // columns (BN/2)*half .. +BN/2-1 of the tile, 64 at a time
         constexpr int kColsPerWarp = BN / 2;
-        uint8_t *patches = smem + Cfg<BN>::kOffPatch + ew * (kPatches * kPatchBytes);
-        float *bias_s = reinterpret_cast<float *>(smem + Cfg<BN>::kOffBias) + ew * kColsPerWarp;
-        int64_t *rowoff = reinterpret_cast<int64_t *>(smem + Cfg<BN>::kOffRowOff) + ew * 32;
+        uint8_t *patches = smem + C::kOffPatch + ew * (kPatches * kPatchBytes);
+        float *bias_s = reinterpret_cast<float *>(smem + C::kOffBias) + ew * kColsPerWarp;
+        int64_t *rowoff = reinterpret_cast<int64_t *>(smem + C::kOffRowOff) + ew * 32;
         const bool scatter = epi.mode == EPI_QKV && epi.paged.slab != nullptr;
         uint32_t pp = 0;                                    // the patch the next staged store fills
         // the store that filled this patch last has read it (the one in flight may still read the other patch)
@@ -180,12 +209,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 else tc::tma_store_2d(map, patch, x, y);
                 tc::bulk_commit();
             }
-            pp ^= 1;
+            pp ^= (uint32_t)(kPatches - 1);
         };
         uint32_t ti = 0;
         bool ok = true;
-        for (int64_t t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++ti) {
-            const int64_t m0 = (t / n_tiles_n) * BM;
+        const uint32_t acc_empty_bar = CTAS == 2 ? tc::cluster_addr(&bars->acc_empty[0], 0) : tc::smem_u32(&bars->acc_empty[0]);
+        for (int64_t t = worker; t < n_tiles && ok; t += n_workers, ++ti) {
+            const int64_t m0 = (t / n_tiles_n) * (BM * CTAS) + rank * BM;
             const int n_w = (int)(t % n_tiles_n) * BN + half * kColsPerWarp;      // first column of this warp's part
             const uint32_t as = ti & 1;
             const int64_t m_base = m0 + quad * 32;
@@ -223,7 +253,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 if (pass == kColsPerWarp / 64 - 1) {
                     tc::tc_fence_before();
                     __syncwarp();
-                    if (lane == 0) tc::mbar_arrive(&bars->acc_empty[as]);      // this warp's part of the accumulator is in registers
+                    if (lane == 0) {                                          // this warp's part of the accumulator is in registers
+                        if constexpr (CTAS == 2) tc::mbar_arrive_cluster(acc_empty_bar + as * 8);
+                        else tc::mbar_arrive(&bars->acc_empty[as]);
+                    }
                 }
                 if (m_base >= M) continue;                                       // the whole row group lies past the last row
                 const int n = n_w + pass * 64;                                   // first output column of these 64
@@ -266,7 +299,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 int which = 0, c = n;                                            // destination tensor and its column
                 if (epi.mode == EPI_QKV) {
                     const int col = epi.col0 + n;
-                    which = col / epi.d_model; c = col - which * epi.d_model;
+                    which = (col >= epi.d_model) + (col >= 2 * epi.d_model); c = col - which * epi.d_model;
                 }
                 const bool paged = paged_tile && which > 0;
                 uint8_t *patch;
@@ -320,26 +353,47 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
     tc::tc_fence_before();
     __syncthreads();
-    if (warp == 1) tc::tmem_dealloc(tmem_base, kTmemCols);
+    if constexpr (CTAS == 2) {
+        tc::cluster_sync();                                       // the peer no longer signals this CTA's barriers or uses its operands
+        if (warp == 1) tc::tmem_dealloc_pair(tmem_base, kTmemCols);
+    } else {
+        if (warp == 1) tc::tmem_dealloc(tmem_base, kTmemCols);
+    }
 }
 
 }  // namespace
 
-template <int BN>
-static cudaError_t launch_bn(const CUtensorMap &tmA, const CUtensorMap &tmB, const GemmOutMaps &om, int64_t M, int N, int K,
-                             const Epilogue &epi, int *err, cudaStream_t stream)
+template <int BN, int CTAS>
+static cudaError_t launch_cfg(const CUtensorMap &tmA, const CUtensorMap &tmB, const GemmOutMaps &om, int64_t M, int N, int K,
+                              const Epilogue &epi, int *err, cudaStream_t stream)
 {
-    static int n_sms = 0;
-    if (n_sms == 0) {
-        int dev = 0;
+    using C = Cfg<BN, CTAS>;
+    static int n_workers_max = 0;                   // CTAs (or CTA pairs) that can be resident at once: one per SM (or SM pair)
+    if (n_workers_max == 0) {
+        int dev = 0, n_sms = 0;
         cudaError_t e = cudaGetDevice(&dev);
         if (e == cudaSuccess) e = cudaDeviceGetAttribute(&n_sms, cudaDevAttrMultiProcessorCount, dev);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_tc_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<BN>::kSmemBytes);
-        if (e != cudaSuccess) { n_sms = 0; return e; }
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_tc_kernel<BN, CTAS>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
+        int n = n_sms / CTAS;
+        if (e == cudaSuccess && CTAS == 2) {
+            cudaLaunchConfig_t cfg{};
+            cfg.gridDim = dim3((unsigned)(2 * n)); cfg.blockDim = dim3(kThreads); cfg.dynamicSmemBytes = C::kSmemBytes;
+            cudaLaunchAttribute attr[1];
+            attr[0].id = cudaLaunchAttributeClusterDimension;
+            attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+            cfg.attrs = attr; cfg.numAttrs = 1;
+            int max_clusters = 0;
+            e = cudaOccupancyMaxActiveClusters(&max_clusters, gemm_tc_kernel<BN, CTAS>, &cfg);
+            if (e == cudaSuccess && max_clusters < n) n = max_clusters;
+        }
+        if (e != cudaSuccess) return e;
+        if (n < 1) return cudaErrorLaunchOutOfResources;
+        n_workers_max = n;
     }
-    const int64_t tiles = ((M + BM - 1) / BM) * (N / BN);
-    const unsigned grid = (unsigned)(tiles < n_sms ? tiles : n_sms);
-    return launch_dependent(gemm_tc_kernel<BN>, dim3(grid), dim3(kThreads), (size_t)Cfg<BN>::kSmemBytes, stream, tmA, tmB, om, M, N, K, epi, err);
+    const int64_t tiles = ((M + BM * CTAS - 1) / (BM * CTAS)) * (N / BN);
+    const unsigned workers = (unsigned)(tiles < n_workers_max ? tiles : n_workers_max);
+    return launch_dependent(gemm_tc_kernel<BN, CTAS>, dim3(workers * CTAS), dim3(kThreads), (size_t)C::kSmemBytes, stream, CTAS, tmA, tmB, om,
+                            M, N, K, epi, err);
 }
 
 cudaError_t launch_gemm_tc(const CUtensorMap &tmA, const CUtensorMap &tmB, const GemmOutMaps &om, int64_t M, int N, int K,
@@ -347,7 +401,8 @@ cudaError_t launch_gemm_tc(const CUtensorMap &tmA, const CUtensorMap &tmB, const
 {
     if (M == 0 || N == 0) return cudaSuccess;
     *launches += 1;
-    return gemm_tile_n(N, K) == 256 ? launch_bn<256>(tmA, tmB, om, M, N, K, epi, err, stream) : launch_bn<128>(tmA, tmB, om, M, N, K, epi, err, stream);
+    return gemm_pair(M, N, K) ? launch_cfg<256, 2>(tmA, tmB, om, M, N, K, epi, err, stream)
+                        : launch_cfg<128, 1>(tmA, tmB, om, M, N, K, epi, err, stream);
 }
 
 }  // namespace relaygr

@@ -12,15 +12,22 @@ namespace relaygr {
 
 // Launch with programmatic stream serialisation: the kernel may begin before its predecessor on the stream has
 // finished, and must call grid_dependency_wait() before reading or writing what earlier kernels produce.
+// cluster_x > 1 launches thread-block clusters of that many CTAs along x (the grid must be a multiple of it).
 template <typename... KArgs, typename... Args>
-cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, Args &&...args)
+cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, int cluster_x,
+                             Args &&...args)
 {
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
+    if (cluster_x > 1) {
+        attr[1].id = cudaLaunchAttributeClusterDimension;
+        attr[1].val.clusterDim.x = (unsigned)cluster_x; attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
+        cfg.numAttrs = 2;
+    }
     return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
 }
 
@@ -62,10 +69,15 @@ cudaError_t launch_attention_simt(const T *q, const T *k_lin, const T *v_lin, Pa
 
 // ---- tensor-core kernels (the bf16 model) -------------------------------------------------------------
 
-// Output tile width of the tensor-core GEMM for [*, K] x [N, K]^T (N % 128 == 0).  A 256-wide tile does twice the MMA
-// work per pipeline hand-shake and per issued instruction, and reads A once per 256 columns; it pays from K = 512 on
-// (measured).  At K = 256 a tile is eight instructions either way and the finer 128-wide tiles balance better.
-inline int gemm_tile_n(int N, int K) { return (N % 256 == 0 && K >= 512) ? 256 : 128; }
+// The tensor-core GEMM for [M, K] x [N, K]^T (N % 128 == 0) runs on CTA pairs (256 x 256 tiles, tcgen05 cta_group::2)
+// when N is a multiple of 256 and the pair's deeper pipeline has enough work to pay for itself: a mainloop of K >= 512,
+// or at least four tiles per pair of SMs (measured on the model's shapes).  Otherwise single CTAs with 128 x 128 tiles.
+// Either way a CTA loads W in boxes of 128 rows.
+inline bool gemm_pair(int64_t M, int N, int K)
+{
+    return N % 256 == 0 && (K >= 512 || ((M + 255) / 256) * (N / 256) >= 4 * 74);
+}
+constexpr int kGemmWeightBoxRows = 128;
 
 // Where a GEMM's epilogue stores: tensor maps with a 32-row box of 128 bytes and the 128-byte swizzle.
 // EPI_STORE: o[0] = out [M, N] bf16.  EPI_RESID: o[0] = the fp32 residual stream [M, N] (tile added in place).
@@ -73,7 +85,7 @@ inline int gemm_tile_n(int N, int K) { return (N % 256 == 0 && K >= 512) ? 256 :
 struct GemmOutMaps { CUtensorMap o[3]; };
 
 // C[m, n] = sum_k A[m, k] W[n, k] on tcgen05; tmA covers A [M, K] with a 128-row box, tmB covers W [N, K]
-// with a box of gemm_tile_n(N, K) rows, both 64 columns wide with the 128-byte swizzle.  N % 128 == 0, K % 64 == 0.
+// with a box of kGemmWeightBoxRows rows, both 64 columns wide with the 128-byte swizzle.  N % 128 == 0, K % 64 == 0.
 // err is a device status word: kernels record a code there instead of hanging or trapping.
 cudaError_t launch_gemm_tc(const CUtensorMap &tmA, const CUtensorMap &tmB, const GemmOutMaps &om, int64_t M, int N, int K,
                            const Epilogue &epi, int *err, cudaStream_t stream, int64_t *launches);

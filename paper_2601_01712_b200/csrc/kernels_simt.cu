@@ -382,7 +382,7 @@ cudaError_t launch_gather_ln(const T *emb, int64_t vocab, int d, RowSource src, 
 {
     if (n_rows == 0) return cudaSuccess;
     *launches += 1;
-    return launch_dependent(gather_ln_kernel<T>, dim3(blocks_for(n_rows)), dim3(kWarpsPerBlock * 32), 0, stream, emb, vocab, d, src, n_rows, g,
+    return launch_dependent(gather_ln_kernel<T>, dim3(blocks_for(n_rows)), dim3(kWarpsPerBlock * 32), 0, stream, 1, emb, vocab, d, src, n_rows, g,
                             b, eps, x, a);
 }
 
@@ -394,7 +394,7 @@ cudaError_t launch_layernorm(const float *x, int d, int64_t n_rows, const float 
     const int nc = (d + 127) / 128;
     cudaError_t e;
 #define RELAYGR_LN(NC, ROWS)                                                                                              \
-    e = launch_dependent(layernorm_kernel<T, NC, ROWS>, dim3(blocks_for((n_rows + ROWS - 1) / ROWS)), dim3(kWarpsPerBlock * 32), 0, stream, \
+    e = launch_dependent(layernorm_kernel<T, NC, ROWS>, dim3(blocks_for((n_rows + ROWS - 1) / ROWS)), dim3(kWarpsPerBlock * 32), 0, stream, 1, \
                          x, d, n_rows, g, b, eps, a)
     if (nc <= 1) RELAYGR_LN(1, 4);
     else if (nc <= 2) RELAYGR_LN(2, 4);
@@ -411,7 +411,7 @@ cudaError_t launch_score(const float *x, int d, const SeqDesc *seqs, int n_users
 {
     if (n_total == 0) return cudaSuccess;
     *launches += 1;
-    return launch_dependent(score_kernel, dim3(blocks_for(n_total)), dim3(kWarpsPerBlock * 32), 0, stream, x, d, seqs, n_users, n_total,
+    return launch_dependent(score_kernel, dim3(blocks_for(n_total)), dim3(kWarpsPerBlock * 32), 0, stream, 1, x, d, seqs, n_users, n_total,
                             score_off, g, b, eps, w, bias, scores);
 }
 
