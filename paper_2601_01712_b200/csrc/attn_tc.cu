@@ -208,6 +208,9 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         const float c = 0.125f * 1.4426950408889634f;        // 1/sqrt(64) * log2(e)
         float m = -INFINITY, l = 0.f;
         bool ok = true;
+        // a warp whose 32 rows all lie past the tile's last row keeps the hand-shakes going but takes no exponentials:
+        // its rows of P (and of O) hold whatever TMEM held, which only ever reaches those same, unused, rows
+        const bool warp_live = quad * 32 < it.n_q;
 
         for (int j = 0; j < nb && ok; ++j) {
             const int blk = it.blk0 + j, b = j & 1;
@@ -221,6 +224,11 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             ok = __all_sync(0xffffffffu, tc::mbar_wait(&bars->s_full[b], (j >> 1) & 1, err));
             if (!ok) break;
             tc::tc_fence_after();
+            if (!warp_live) {
+                tc::tc_fence_before();
+                tc::mbar_arrive(&bars->p_full[b]);
+                continue;
+            }
 
             // the S row of this block, in registers
             uint32_t s0[32], s1[32];
@@ -313,7 +321,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         // ---- epilogue: O / l (plus the candidate's own key), or the split partial
         if (ok && nb > 0) ok = __all_sync(0xffffffffu, tc::mbar_wait(&bars->p_free[(nb - 1) & 1], ((nb - 1) >> 1) & 1, err));
         tc::tc_fence_after();
-        if (ok) {
+        if (ok && warp_live) {
             float o[kDh];
             if (nb > 0) {
 #pragma unroll

@@ -232,7 +232,14 @@ int Forward::run_t(const CallDesc &call, float *scores, cudaStream_t stream, std
         const int64_t target = 2 * (int64_t)n_sms;
         int want = base > 0 && base < target ? (int)((target + base - 1) / base) : 1;
         int part_slot = 0;
-        std::sort(tiles.begin(), tiles.end(), [](const Tile &x, const Tile &y) { return x.nb > y.nb; });   // longest first
+        // costliest first (key blocks x softmax warps with live rows), so that the cheap partial tiles fill the last wave;
+        // ties keep a user's tiles together (they share K / V through L2)
+        std::sort(tiles.begin(), tiles.end(), [](const Tile &x, const Tile &y) {
+            const int64_t cx = (int64_t)x.nb * ((x.n_q + 31) / 32), cy = (int64_t)y.nb * ((y.n_q + 31) / 32);
+            if (cx != cy) return cx > cy;
+            if (x.seq != y.seq) return x.seq < y.seq;
+            return x.q0 < y.q0;
+        });
         for (const Tile &t : tiles) {
             int ns = std::max(1, std::min(want, t.nb / 8));          // at least 8 key blocks (512 keys) per split
             if (ns > 1 && part_slot + ns * H > kMaxSplitTiles) ns = 1;
