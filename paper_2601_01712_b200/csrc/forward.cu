@@ -307,8 +307,12 @@ int Forward::run_t(const CallDesc &call, float *scores, cudaStream_t stream, std
         trc |= make_tmap_2d_bf16(&om_qkv.o[2], vl, (uint64_t)R, (uint64_t)d, (uint64_t)d, 32, 64);
         trc |= make_tmap_2d_bf16(&om_hid.o[0], hid, (uint64_t)R, (uint64_t)F, (uint64_t)F, 32, 64);
         trc |= make_tmap_2d_f32(&om_x.o[0], x, (uint64_t)R, (uint64_t)d, (uint64_t)d, 32, 32);
-        om_hid.o[1] = om_hid.o[2] = om_hid.o[0];
-        om_x.o[1] = om_x.o[2] = om_x.o[0];
+        if (call.pool_slab)
+            trc |= make_tmap_2d_bf16(&om_qkv.pool, call.pool_slab, (uint64_t)call.pool_pages * L * 2 * 64, (uint64_t)d, (uint64_t)d, 32, 64);
+        else
+            om_qkv.pool = om_qkv.o[0];
+        om_hid.o[1] = om_hid.o[2] = om_hid.pool = om_hid.o[0];
+        om_x.o[1] = om_x.o[2] = om_x.pool = om_x.o[0];
         if (trc != 0) { err = "tensor-map encoding of the activations failed"; return RELAYGR_E_CUDA; }
     }
     auto gemm = [&](const T *A, const CUtensorMap &tmA, const T *W, const CUtensorMap *tmW, const GemmOutMaps &om, int N, int K,

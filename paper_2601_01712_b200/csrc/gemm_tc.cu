@@ -228,16 +228,22 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             }
             int last_slot = -1, page = 0;
             const bool paged_tile = scatter && epi.col0 + n_w + kColsPerWarp - 1 >= epi.d_model;
+            bool run = false;                               // the warp's 32 rows are 32 consecutive slots of one page
+            int pool_row0 = 0;                              // row of (page, K, first slot) in the pool map; V is 64 rows on
             if (paged_tile) {
                 int64_t off = 0;
+                int u = -1, tt = 0;
                 if (m < M) {
-                    const int u = find_user(epi.row_off, epi.n_users, (int)m);
-                    const int tt = (int)m - epi.row_off[u];
+                    u = find_user(epi.row_off, epi.n_users, (int)m);
+                    tt = (int)m - epi.row_off[u];
                     page = epi.paged.pt[epi.seqs[u].pt_base + (tt >> 6)];
                     off = (int64_t)page_elem_offset(epi.paged, page, 0, tt & 63);
                     if (tt == epi.seqs[u].n_q - 1) last_slot = tt & 63;
                 }
                 rowoff[lane] = off;
+                const int u0 = __shfl_sync(0xffffffffu, u, 0), tt0 = __shfl_sync(0xffffffffu, tt, 0), page0 = __shfl_sync(0xffffffffu, page, 0);
+                run = __all_sync(0xffffffffu, u >= 0 && u == u0 && tt == tt0 + lane && (tt0 & 63) <= 32);
+                pool_row0 = ((page0 * epi.paged.n_layers + epi.paged.layer) * 2) * 64 + (tt0 & 63);
             }
             __syncwarp();
             ok = __all_sync(0xffffffffu, tc::mbar_wait(&bars->acc_full[as], (ti >> 1) & 1, err));
@@ -303,8 +309,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 }
                 const bool paged = paged_tile && which > 0;
                 uint8_t *patch;
-                if (paged) {
-                    if (lane == 0) tc::bulk_wait_read<0>();                      // both patches idle: this path reads its own staging
+                if (paged && !run) {
+                    if (lane == 0) tc::bulk_wait_read<0>();                      // the patches are idle: this path reads its own staging
                     __syncwarp();
                     patch = patches;
                 } else {
@@ -327,6 +333,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     patch_submit(&om.o[which], patch, c, (int)m_base, false);
                     continue;
                 }
+                if (run) {
+                    // the 32 rows are consecutive slots of one page: one bulk tensor store into the pool
+                    patch_submit(&om.pool, patch, c, pool_row0 + (which - 1) * 64, false);
+                } else {
                 // K / V rows into pages: 8 lanes per row copy its 128 bytes to (page, K | V, slot)
                 __syncwarp();
                 __nv_bfloat16 *kv = reinterpret_cast<__nv_bfloat16 *>(epi.paged.slab) + (size_t)(which - 1) * 64 * epi.d_model + c;
@@ -337,6 +347,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     if (m_base + r < M) *reinterpret_cast<uint4 *>(kv + rowoff[r] + cj * 8) = *patch_chunk(patch, r, cj);
                 }
                 __syncwarp();
+                }
                 if (last_slot >= 0 && last_slot < 63) {
                     // last prefix row of a user: clear the unused slots of its last page (they are masked, but must hold finite values)
                     __nv_bfloat16 *slab = reinterpret_cast<__nv_bfloat16 *>(epi.paged.slab);

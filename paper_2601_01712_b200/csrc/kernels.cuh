@@ -81,8 +81,9 @@ constexpr int kGemmWeightBoxRows = 128;
 
 // Where a GEMM's epilogue stores: tensor maps with a 32-row box of 128 bytes and the 128-byte swizzle.
 // EPI_STORE: o[0] = out [M, N] bf16.  EPI_RESID: o[0] = the fp32 residual stream [M, N] (tile added in place).
-// EPI_QKV: o[0] = q, o[1] = k_lin, o[2] = v_lin, each [M, d] bf16 (o[1], o[2] are not used when K / V go to pages).
-struct GemmOutMaps { CUtensorMap o[3]; };
+// EPI_QKV: o[0] = q, o[1] = k_lin, o[2] = v_lin, each [M, d] bf16 (o[1], o[2] are not used when K / V go to pages);
+// pool = the pool slab viewed as [pages * L * 2 * 64, d] (used when K / V go to pages, else any valid map).
+struct GemmOutMaps { CUtensorMap o[3]; CUtensorMap pool; };
 
 // C[m, n] = sum_k A[m, k] W[n, k] on tcgen05; tmA covers A [M, K] with a 128-row box, tmB covers W [N, K]
 // with a box of kGemmWeightBoxRows rows, both 64 columns wide with the 128-byte swizzle.  N % 128 == 0, K % 64 == 0.
