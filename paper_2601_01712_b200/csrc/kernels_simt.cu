@@ -398,7 +398,7 @@ cudaError_t launch_layernorm(const float *x, int d, int64_t n_rows, const float 
                          x, d, n_rows, g, b, eps, a)
     if (nc <= 1) RELAYGR_LN(1, 4);
     else if (nc <= 2) RELAYGR_LN(2, 4);
-    else if (nc <= 4) RELAYGR_LN(4, 2);
+    else if (nc <= 4) RELAYGR_LN(4, 4);
     else RELAYGR_LN(8, 1);
 #undef RELAYGR_LN
     *launches += 1;
