@@ -20,7 +20,7 @@ _LIB = os.path.join(_HERE, "librelaygr_oracle.so")
 
 class _Cfg(C.Structure):
     _fields_ = [("n_layers", C.c_int32), ("d_model", C.c_int32), ("n_heads", C.c_int32),
-                ("d_head", C.c_int32), ("d_ff", C.c_int32), ("ln_eps", C.c_double)]
+                ("d_head", C.c_int32), ("d_ff", C.c_int32), ("ln_eps", C.c_double), ("attn_kind", C.c_int32)]
 
 
 _WNAMES = ["emb", "ln1_g", "ln1_b", "ln2_g", "ln2_b", "w_qkv", "b_qkv", "w_o", "b_o",
@@ -68,13 +68,14 @@ class Model:
 
     ``params`` maps the names emb, ln1_g, ln1_b, ln2_g, ln2_b, w_qkv, b_qkv,
     w_o, b_o, w1, b1, w2, b2, lnf_g, lnf_b, w_score, b_score to fp32 arrays;
-    linear weights are ``[L, out, in]``; a bias may be ``None``.
+    linear weights are ``[L, out, in]``; a bias may be ``None``.  ``attn_kind``: 0 softmax attention,
+    1 pointwise SiLU attention (the checker's header states both).
     """
 
     def __init__(self, n_layers: int, d_model: int, n_heads: int, d_head: int, d_ff: int,
-                 ln_eps: float, params: Dict[str, Optional[np.ndarray]]):
-        assert n_heads * d_head == d_model
-        self.cfg = _Cfg(n_layers, d_model, n_heads, d_head, d_ff, float(ln_eps))
+                 ln_eps: float, params: Dict[str, Optional[np.ndarray]], attn_kind: int = 0):
+        assert n_heads * d_head == d_model and attn_kind in (0, 1)
+        self.cfg = _Cfg(n_layers, d_model, n_heads, d_head, d_ff, float(ln_eps), int(attn_kind))
         self.L, self.d = n_layers, d_model
         self._keep = {}
         self.w = _W()

@@ -20,6 +20,17 @@
  *   so the prefix is item-independent (Section 3.1) and candidates never see
  *   one another.
  *
+ *   attn_kind selects how the allowed keys are aggregated:
+ *     0  softmax attention      o_t = sum_j softmax_j(q_t.k_j / sqrt(dh)) v_j
+ *     1  pointwise aggregated attention in the style of HSTU, the model family
+ *        the paper's evaluation names (Section 5.1): the softmax is replaced by
+ *        an elementwise SiLU, o_t = (1 / |A(t)|) sum_j SiLU(q_t.k_j / sqrt(dh)) v_j.
+ *        Readings: HSTU's relative attention bias is left out (no positions or
+ *        timestamps exist in this model), the logit scale 1/sqrt(dh) is kept
+ *        from the softmax block, and the normaliser is the number of keys the
+ *        query may see (HSTU divides by the sequence length).  Only the
+ *        attention changes; the block around it stays the pre-LN transformer.
+ *
  *   orc_full        f([U,S_l,S~_l,I], {})  - one pass over all P+S+C tokens.
  *   orc_preinfer    psi <- f([U,S_l,{},{}], {}) - prefix only, returns the
  *                   per-layer K and V rows (Section 2.3, Section 4.1 "cache
@@ -46,6 +57,7 @@
 typedef struct {
     int32_t n_layers, d_model, n_heads, d_head, d_ff;
     double ln_eps;
+    int32_t attn_kind;                              /* 0 softmax, 1 pointwise SiLU (see above) */
 } orc_cfg;
 
 /* Linear weights are [out, in] row-major: y = x W^T + b. */
@@ -129,7 +141,8 @@ static void block(const orc_cfg *c, const orc_weights *w, int l, int64_t P, int6
         }
     }
 
-    /* o_t = sum_{j in A(t)} softmax_j(q_t . k_j / sqrt(dh)) v_j, per head */
+    /* o_t = sum_{j in A(t)} softmax_j(q_t . k_j / sqrt(dh)) v_j, per head;
+     * or, attn_kind 1, o_t = (1 / |A(t)|) sum_{j in A(t)} SiLU(q_t . k_j / sqrt(dh)) v_j */
     const double scale = 1.0 / sqrt((double)dh);
     const int64_t n_keys = n_ctx + n;
 #pragma omp parallel for schedule(dynamic, 4)
@@ -138,6 +151,24 @@ static void block(const orc_cfg *c, const orc_weights *w, int l, int64_t P, int6
         const int64_t tpos = pos0 + t;
         for (int h = 0; h < H; ++h) {
             const double *q = qkv + t * 3 * d + h * dh;
+            if (c->attn_kind == 1) {
+                double *o = att + t * d + h * dh;
+                for (int e = 0; e < dh; ++e) o[e] = 0.0;
+                int64_t n_seen = 0;
+                for (int64_t j = 0; j < n_keys; ++j) {
+                    const int64_t jpos = j < n_ctx ? j : pos0 + (j - n_ctx);
+                    if (!allowed(P, S, tpos, jpos)) continue;
+                    const double *k = j < n_ctx ? Kctx + j * d + h * dh : qkv + (j - n_ctx) * 3 * d + d + h * dh;
+                    const double *v = j < n_ctx ? Vctx + j * d + h * dh : qkv + (j - n_ctx) * 3 * d + 2 * d + h * dh;
+                    double dot = 0.0;
+                    for (int e = 0; e < dh; ++e) dot += q[e] * k[e];
+                    const double p = silu(dot * scale);
+                    for (int e = 0; e < dh; ++e) o[e] += p * v[e];
+                    ++n_seen;
+                }
+                for (int e = 0; e < dh; ++e) o[e] /= (double)n_seen;     /* a query always sees itself */
+                continue;
+            }
             double m = -INFINITY;
             for (int64_t j = 0; j < n_keys; ++j) {
                 const int64_t jpos = j < n_ctx ? j : pos0 + (j - n_ctx);

@@ -42,6 +42,7 @@ class ModelShape:
     dtype: int
     ln_eps: float = 1e-5
     page_tokens: int = PAGE_TOKENS
+    attn_kind: int = 0            # 0 softmax attention, 1 pointwise SiLU attention (HSTU style)
 
     def kv_bytes(self, prefix_len: int) -> int:
         """Bytes of per-layer K and V kept for a prefix of ``prefix_len`` tokens."""

@@ -2,8 +2,10 @@
 
 A second, independent writing of the model used only to pin the CPU checker on
 tiny inputs: it materialises the full (P+S+C)^2 boolean mask and evaluates
-softmax(Q K^T / sqrt(d_h) + mask) V head by head.  It shares no code with the
-checker in ``oracle/`` or with the CUDA library.
+softmax(Q K^T / sqrt(d_h) + mask) V head by head - or, for the pointwise
+variant (``shape["attn_kind"] == 1``), (SiLU(Q K^T / sqrt(d_h)) * mask) V divided
+by each row's count of visible keys.  It shares no code with the checker in
+``oracle/`` or with the CUDA library.
 """
 import numpy as np
 
@@ -44,6 +46,10 @@ def forward(shape, w, ids_all, mask):
         for h in range(H):
             sl = slice(h * dh, (h + 1) * dh)
             s = q[:, sl] @ k[:, sl].T / np.sqrt(dh)
+            if shape.get("attn_kind", 0) == 1:
+                p = np.where(mask, s / (1.0 + np.exp(-s)), 0.0)
+                att[:, sl] = (p @ v[:, sl]) / mask.sum(axis=1, keepdims=True)
+                continue
             s = np.where(mask, s, -np.inf)
             s = s - s.max(axis=1, keepdims=True)
             p = np.exp(s)
