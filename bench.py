@@ -136,6 +136,8 @@ def main():
     ap.add_argument("--candidates", type=int, default=0, help="candidates per user (0 = the workload's own: 512, or 1024 for workload 4)")
     ap.add_argument("--layers", type=int, default=0, help="override the model's depth (sweeps)")
     ap.add_argument("--d-model", type=int, default=0, help="override the model's width (heads of 64, FFN 4x; sweeps)")
+    ap.add_argument("--attention", default="softmax", choices=["softmax", "pointwise"],
+                    help="pointwise: the HSTU-style SiLU attention variant of the same model (sweeps)")
     args = ap.parse_args()
     if args.impl == "reference":
         return reference_arm(args)
@@ -159,10 +161,13 @@ def main():
 
     wl = synth.workload(args.workload)
     shape = wl.model
-    if args.layers or args.d_model:
+    pointwise = args.attention == "pointwise"
+    if args.layers or args.d_model or pointwise:
         dm = args.d_model or shape.d_model
-        shape = synth.ModelShape(args.layers or shape.n_layers, dm, dm // 64, 64, 4 * dm, shape.vocab, shape.dtype)
-    custom = ("; overrides: layers %d, d_model %d" % (shape.n_layers, shape.d_model)) if (args.layers or args.d_model) else ""
+        shape = synth.ModelShape(args.layers or shape.n_layers, dm, dm // 64, 64, 4 * dm, shape.vocab, shape.dtype,
+                                 attn_kind=1 if pointwise else 0)
+    custom = ("; overrides: layers %d, d_model %d%s" % (shape.n_layers, shape.d_model, ", pointwise SiLU attention" if pointwise else "")) \
+        if (args.layers or args.d_model or pointwise) else ""
     if args.workload == 3:
         n_users = args.users or 128
         pl, sl, cl = synth.config3_lengths(np.random.default_rng(wl.seed + 1000 * rank), n_users)

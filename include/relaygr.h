@@ -84,13 +84,25 @@ typedef struct relaygr_kv_pool relaygr_kv_pool;
  *   F32 : any d_model multiple of 4, d_head in {32, 64}        (CUDA-core kernels)
  *   BF16: d_head = 64, d_model and d_ff multiples of 128       (tcgen05 kernels)
  * page_tokens must be 64.
+ *
+ * attn_kind selects how a query aggregates the keys it may see (the mask is the same):
+ *   RELAYGR_ATTN_SOFTMAX    o_t = sum_j softmax_j(q_t.k_j / sqrt(d_head)) v_j - the block the evaluation
+ *                           configurations name.
+ *   RELAYGR_ATTN_POINTWISE  o_t = (1 / n_t) sum_j SiLU(q_t.k_j / sqrt(d_head)) v_j, n_t = number of keys visible to t:
+ *                           the pointwise aggregated attention of HSTU, the model family of the paper's
+ *                           evaluation (Section 5.1), without its relative attention bias.  Everything else
+ *                           (the mask, the K/V pool, rank on cache == full inference) is unchanged.
  */
+#define RELAYGR_ATTN_SOFTMAX   0
+#define RELAYGR_ATTN_POINTWISE 1
+
 typedef struct {
     int32_t n_layers, d_model, n_heads, d_head, d_ff;
     int32_t dtype;
     int32_t page_tokens;
     int64_t vocab;
     float ln_eps;
+    int32_t attn_kind;   /* RELAYGR_ATTN_*; zero (softmax) when the struct is zero-initialised */
 } relaygr_model_cfg;
 
 /*

@@ -23,7 +23,7 @@ STATUS_NAMES = {0: "OK", -1: "E_INVALID", -2: "E_NOSPACE", -3: "E_EXISTS", -4: "
 class ModelCfg(C.Structure):
     _fields_ = [("n_layers", C.c_int32), ("d_model", C.c_int32), ("n_heads", C.c_int32), ("d_head", C.c_int32),
                 ("d_ff", C.c_int32), ("dtype", C.c_int32), ("page_tokens", C.c_int32), ("vocab", C.c_int64),
-                ("ln_eps", C.c_float)]
+                ("ln_eps", C.c_float), ("attn_kind", C.c_int32)]
 
 
 WEIGHT_FIELDS = ["emb", "ln1_g", "ln1_b", "ln2_g", "ln2_b", "w_qkv", "b_qkv", "w_o", "b_o", "w1", "b1", "w2", "b2",

@@ -77,6 +77,9 @@ __device__ __forceinline__ float max3(float a, float b, float c)
     return d;
 }
 
+// kPointwise: pointwise aggregated attention (HSTU style) - the weight of a visible key is SiLU(q.k / sqrt(d_h)) and the
+// sum is divided by the number of visible keys; no running maximum, no row sum, no rescaling of O.
+template <bool kPointwise>
 __global__ void __launch_bounds__(192, 2)
 attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmKlin,
                     const __grid_constant__ CUtensorMap tmVlin, const __grid_constant__ CUtensorMap tmPool,
@@ -238,9 +241,33 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             if (need_mask) {
 #pragma unroll
                 for (int i = 0; i < 32; ++i) {
-                    if (i >= jmax) s0[i] = 0xff800000u;      // -inf
-                    if (32 + i >= jmax) s1[i] = 0xff800000u;
+                    if (i >= jmax) s0[i] = kPointwise ? 0u : 0xff800000u;      // -inf (softmax) or a logit of 0: SiLU(0) = 0
+                    if (32 + i >= jmax) s1[i] = kPointwise ? 0u : 0xff800000u;
                 }
+            }
+            if constexpr (kPointwise) {
+                // p = SiLU(z) = h + h tanh(h), h = z / 2, z = s / sqrt(d_h): one MUFU op per key, bf16 P into TMEM
+                const uint64_t hc2 = pack2(0.0625f, 0.0625f), zero2 = pack2(0.f, 0.f);
+                uint32_t pk[16];
+#pragma unroll
+                for (int half = 0; half < 2; ++half) {
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        const uint32_t a0 = half == 0 ? s0[2 * i] : s1[2 * i], a1 = half == 0 ? s0[2 * i + 1] : s1[2 * i + 1];
+                        float h0, h1, t0, t1, p0, p1;
+                        const uint64_t h2 = fma2(pack2(__uint_as_float(a0), __uint_as_float(a1)), hc2, zero2);
+                        unpack2(h2, h0, h1);
+                        asm("tanh.approx.f32 %0, %1;" : "=f"(t0) : "f"(h0));
+                        asm("tanh.approx.f32 %0, %1;" : "=f"(t1) : "f"(h1));
+                        unpack2(fma2(h2, pack2(t0, t1), h2), p0, p1);
+                        pk[i] = tc::pack_bf16(p0, p1);
+                    }
+                    tc::tmem_st16(lane_addr + kColP + b * (kKeys / 2) + 16 * half, pk);
+                }
+                tc::tmem_st_wait();
+                tc::tc_fence_before();
+                tc::mbar_arrive(&bars->p_full[b]);
+                continue;
             }
             // p = 2^(s c - m c), bf16 P into TMEM (P[b] is free: see the MMA issuer), row sum in fp32.  The exponentials
             // are first taken against the running maximum as it stood before this block; only if the row sum shows that
@@ -355,11 +382,18 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                         dot = fmaf(fa.x, fb.x, dot); dot = fmaf(fa.y, fb.y, dot);
                     }
                 }
-                const float mn = fmaxf(m, dot);
-                const float al = (m == -INFINITY) ? 0.f : ex2((m - mn) * c);
-                const float ps = ex2((dot - mn) * c);
-                l = l * al + ps;
-                m = mn;
+                float al, ps;
+                if constexpr (kPointwise) {
+                    const float z = dot * 0.125f;
+                    al = 1.f;
+                    ps = z / (1.f + __expf(-z));
+                } else {
+                    const float mn = fmaxf(m, dot);
+                    al = (m == -INFINITY) ? 0.f : ex2((m - mn) * c);
+                    ps = ex2((dot - mn) * c);
+                    l = l * al + ps;
+                    m = mn;
+                }
 #pragma unroll
                 for (int i = 0; i < 8; ++i) {
                     const uint4 vv = vp[i];
@@ -371,6 +405,13 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                         o[i * 8 + 2 * e + 1] = fmaf(o[i * 8 + 2 * e + 1], al, ps * fv.y);
                     }
                 }
+            }
+            if constexpr (kPointwise) {
+                // the normaliser is the number of keys the row may see (every key position below its limit, plus itself for
+                // a candidate); a split item hands it over as l with m = 0, so that the merge of partials needs no change
+                const float n_seen = (float)(is_cand ? sd.causal_end + 1 : tpos + 1);
+                m = 0.f;
+                l = (it.partial_slot < 0 || it.blk0 == 0) ? n_seen : 0.f;
             }
             if (row_ok) {
                 if (it.partial_slot < 0) {
@@ -436,18 +477,20 @@ attention_merge_kernel(const AttnMerge *__restrict__ merges, const SeqDesc *__re
 cudaError_t launch_attention_tc(const CUtensorMap &tmQ, const CUtensorMap &tmK, const CUtensorMap &tmV, const CUtensorMap &tmPool,
                                 const AttnItem *items, int n_items, const AttnMerge *merges, int n_merges, const SeqDesc *seqs,
                                 const int32_t *pt, int n_layers, int layer, int d_model, const __nv_bfloat16 *q,
-                                const __nv_bfloat16 *k_lin, const __nv_bfloat16 *v_lin, __nv_bfloat16 *out, float *partial,
-                                int *err, cudaStream_t stream, int64_t *launches)
+                                const __nv_bfloat16 *k_lin, const __nv_bfloat16 *v_lin, int attn_kind, __nv_bfloat16 *out,
+                                float *partial, int *err, cudaStream_t stream, int64_t *launches)
 {
     if (n_items == 0) return cudaSuccess;
     static bool attr_set = false;
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        cudaError_t e = cudaFuncSetAttribute(attention_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(attention_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
     *launches += 1;
-    cudaError_t e = launch_dependent(attention_tc_kernel, dim3(n_items), dim3(192), (size_t)kSmemBytes, stream, 1, tmQ, tmK, tmV, tmPool, items,
+    auto kernel = attn_kind == ATTN_POINTWISE ? attention_tc_kernel<true> : attention_tc_kernel<false>;
+    cudaError_t e = launch_dependent(kernel, dim3(n_items), dim3(192), (size_t)kSmemBytes, stream, 1, tmQ, tmK, tmV, tmPool, items,
                                      seqs, pt, n_layers, layer, d_model, q, k_lin, v_lin, out, partial, err);
     if (e != cudaSuccess || n_merges == 0) return e;
     *launches += 1;

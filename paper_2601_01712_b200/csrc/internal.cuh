@@ -54,6 +54,9 @@ struct AttnMerge {
 
 enum EpiMode : int32_t { EPI_STORE = 0, EPI_RESID = 1, EPI_QKV = 2 };
 
+// How a query aggregates the keys it may see (relaygr_model_cfg.attn_kind).
+enum AttnKind : int32_t { ATTN_SOFTMAX = 0, ATTN_POINTWISE = 1 };
+
 // What a GEMM does with its fp32 accumulators: C[m, n] = sum_k A[m,k] W[n,k].
 struct Epilogue {
     int32_t mode;

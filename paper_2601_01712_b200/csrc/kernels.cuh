@@ -61,10 +61,10 @@ template <typename T>
 cudaError_t launch_gemm_simt(const T *A, const T *W, int64_t M, int N, int K, const Epilogue &epi,
                              cudaStream_t stream, int64_t *launches);
 
-// One warp per (row, head): softmax attention under the SeqDesc mask.  out [n_rows, d] in T.
+// One warp per (row, head): attention (softmax, or pointwise SiLU for ATTN_POINTWISE) under the SeqDesc mask.  out [n_rows, d] in T.
 template <typename T>
 cudaError_t launch_attention_simt(const T *q, const T *k_lin, const T *v_lin, PagedKV paged, const SeqDesc *seqs,
-                                  const int32_t *row_off, int n_users, int64_t n_rows, int n_heads, int d_head,
+                                  const int32_t *row_off, int n_users, int64_t n_rows, int n_heads, int d_head, int attn_kind,
                                   T *out, cudaStream_t stream, int64_t *launches);
 
 // ---- tensor-core kernels (the bf16 model) -------------------------------------------------------------
@@ -91,13 +91,14 @@ struct GemmOutMaps { CUtensorMap o[3]; CUtensorMap pool; };
 cudaError_t launch_gemm_tc(const CUtensorMap &tmA, const CUtensorMap &tmB, const GemmOutMaps &om, int64_t M, int N, int K,
                            const Epilogue &epi, int *err, cudaStream_t stream, int64_t *launches);
 
-// Flash-style attention on tcgen05 (d_head = 64) over the work items, then the merge of split items.
+// Flash-style attention on tcgen05 (d_head = 64) over the work items, then the merge of split items.  attn_kind: ATTN_SOFTMAX, or
+// ATTN_POINTWISE (weights SiLU(q.k / sqrt(d_h)) divided by the number of visible keys).
 // tmQ: [rows, d] box 128 x 64; tmK / tmV: the call's transient K / V rows, box 64 x 64; tmPool: the pool
 // slab viewed as [pages * L * 2 * 64, d], box 64 x 64 (pass tmK when the call has no pool).
 cudaError_t launch_attention_tc(const CUtensorMap &tmQ, const CUtensorMap &tmK, const CUtensorMap &tmV, const CUtensorMap &tmPool,
                                 const AttnItem *items, int n_items, const AttnMerge *merges, int n_merges, const SeqDesc *seqs,
                                 const int32_t *pt, int n_layers, int layer, int d_model, const __nv_bfloat16 *q,
-                                const __nv_bfloat16 *k_lin, const __nv_bfloat16 *v_lin, __nv_bfloat16 *out, float *partial,
-                                int *err, cudaStream_t stream, int64_t *launches);
+                                const __nv_bfloat16 *k_lin, const __nv_bfloat16 *v_lin, int attn_kind, __nv_bfloat16 *out,
+                                float *partial, int *err, cudaStream_t stream, int64_t *launches);
 
 }  // namespace relaygr

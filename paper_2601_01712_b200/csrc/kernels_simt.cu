@@ -307,7 +307,7 @@ template <typename T, int DH>
 __global__ void __launch_bounds__(kWarpsPerBlock * 32)
 attention_simt_kernel(const T *__restrict__ q, const T *__restrict__ k_lin, const T *__restrict__ v_lin, PagedKV paged,
                       const SeqDesc *__restrict__ seqs, const int32_t *__restrict__ row_off, int n_users, int64_t n_rows,
-                      int n_heads, T *__restrict__ out)
+                      int n_heads, int attn_kind, T *__restrict__ out)
 {
     constexpr int PER = DH / 32;
     const int64_t wid = (int64_t)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
@@ -332,6 +332,14 @@ attention_simt_kernel(const T *__restrict__ q, const T *__restrict__ k_lin, cons
 #pragma unroll
         for (int i = 0; i < PER; ++i) dot += qv[i] * Num<T>::to_f(kp[lane * PER + i]);
         dot = warp_sum(dot);
+        if (attn_kind == ATTN_POINTWISE) {
+            // pointwise aggregation: weight SiLU(logit), normalised by the number of visible keys (counted in l)
+            const float p = dot / (1.f + expf(-dot));
+            l += 1.f;
+#pragma unroll
+            for (int i = 0; i < PER; ++i) o[i] += p * Num<T>::to_f(vp[lane * PER + i]);
+            return;
+        }
         const float mn = fmaxf(m, dot);
         const float corr = expf(m - mn), p = expf(dot - mn);
         l = l * corr + p;
@@ -428,17 +436,17 @@ cudaError_t launch_gemm_simt(const T *A, const T *W, int64_t M, int N, int K, co
 
 template <typename T>
 cudaError_t launch_attention_simt(const T *q, const T *k_lin, const T *v_lin, PagedKV paged, const SeqDesc *seqs,
-                                  const int32_t *row_off, int n_users, int64_t n_rows, int n_heads, int d_head, T *out,
-                                  cudaStream_t stream, int64_t *launches)
+                                  const int32_t *row_off, int n_users, int64_t n_rows, int n_heads, int d_head, int attn_kind,
+                                  T *out, cudaStream_t stream, int64_t *launches)
 {
     if (n_rows == 0) return cudaSuccess;
     const unsigned blocks = blocks_for(n_rows * n_heads);
     if (d_head == 32)
         attention_simt_kernel<T, 32><<<blocks, kWarpsPerBlock * 32, 0, stream>>>(q, k_lin, v_lin, paged, seqs, row_off, n_users,
-                                                                                 n_rows, n_heads, out);
+                                                                                 n_rows, n_heads, attn_kind, out);
     else if (d_head == 64)
         attention_simt_kernel<T, 64><<<blocks, kWarpsPerBlock * 32, 0, stream>>>(q, k_lin, v_lin, paged, seqs, row_off, n_users,
-                                                                                 n_rows, n_heads, out);
+                                                                                 n_rows, n_heads, attn_kind, out);
     else
         return cudaErrorInvalidValue;
     *launches += 1;
@@ -454,7 +462,7 @@ cudaError_t launch_attention_simt(const T *q, const T *k_lin, const T *v_lin, Pa
     template cudaError_t launch_gemm_simt<T>(const T *, const T *, int64_t, int, int, const Epilogue &, cudaStream_t,        \
                                              int64_t *);                                                                    \
     template cudaError_t launch_attention_simt<T>(const T *, const T *, const T *, PagedKV, const SeqDesc *, const int32_t *, \
-                                                  int, int64_t, int, int, T *, cudaStream_t, int64_t *);
+                                                  int, int64_t, int, int, int, T *, cudaStream_t, int64_t *);
 RELAYGR_INSTANTIATE(float)
 RELAYGR_INSTANTIATE(__nv_bfloat16)
 

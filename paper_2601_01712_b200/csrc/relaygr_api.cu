@@ -54,6 +54,8 @@ static int check_cfg(const relaygr_model_cfg *c)
         return fail(RELAYGR_E_INVALID, "model sizes must be positive");
     if (c->n_heads * c->d_head != c->d_model) return fail(RELAYGR_E_INVALID, "d_model must equal n_heads * d_head");
     if (c->page_tokens != 64) return fail(RELAYGR_E_UNSUPPORTED, "page_tokens must be 64");
+    if (c->attn_kind != RELAYGR_ATTN_SOFTMAX && c->attn_kind != RELAYGR_ATTN_POINTWISE)
+        return fail(RELAYGR_E_INVALID, "attn_kind must be RELAYGR_ATTN_SOFTMAX or RELAYGR_ATTN_POINTWISE");
     if (c->d_model > 1024) return fail(RELAYGR_E_UNSUPPORTED, "d_model above 1024 is not supported");
     if (c->dtype == RELAYGR_DTYPE_F32) {
         if (c->d_model % 4 || c->d_ff % 4) return fail(RELAYGR_E_UNSUPPORTED, "fp32 model: d_model and d_ff must be multiples of 4");
@@ -289,7 +291,7 @@ static bool same_model(const relaygr_ctx *a, const relaygr_ctx *b)
 {
     const relaygr_model_cfg &x = a->fwd.cfg, &y = b->fwd.cfg;
     return a == b || (x.n_layers == y.n_layers && x.d_model == y.d_model && x.n_heads == y.n_heads && x.d_head == y.d_head &&
-                      x.d_ff == y.d_ff && x.dtype == y.dtype && x.page_tokens == y.page_tokens && x.vocab == y.vocab &&
+                      x.d_ff == y.d_ff && x.dtype == y.dtype && x.page_tokens == y.page_tokens && x.vocab == y.vocab && x.attn_kind == y.attn_kind &&
                       a->host_only == b->host_only && a->fwd.w.w_qkv == b->fwd.w.w_qkv && a->fwd.w.emb == b->fwd.w.emb);
 }
 

@@ -37,7 +37,7 @@ class Model:
         for name, a in weights.vec.items():
             self._t[name] = torch.from_numpy(a).to(self.device).contiguous()
         self.cfg = B.ModelCfg(shape.n_layers, shape.d_model, shape.n_heads, shape.d_head, shape.d_ff, shape.dtype,
-                              shape.page_tokens, weights.mat["emb"].shape[0], shape.ln_eps)
+                              shape.page_tokens, weights.mat["emb"].shape[0], shape.ln_eps, shape.attn_kind)
         w = B.Weights()
         for name in B.WEIGHT_FIELDS:
             setattr(w, name, self._t[name].data_ptr())

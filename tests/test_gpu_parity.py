@@ -6,7 +6,7 @@ import pytest
 import torch
 
 from paper_2601_01712_b200 import synth
-from tests.helpers import TOL_BF16, TOL_F32, max_abs_err, oracle_model, oracle_scores, small_bf16_shape
+from tests.helpers import TOL_BF16, TOL_BF16_POINTWISE, TOL_F32, max_abs_err, oracle_model, oracle_scores, small_bf16_shape
 
 pytestmark = pytest.mark.gpu
 
@@ -375,5 +375,67 @@ def test_degenerate_batches():
     want = oracle_scores(om, batch)
     assert max_abs_err(scores, batch, want) <= TOL_BF16
     assert max_abs_err(full, batch, want) <= TOL_BF16
+    assert model.device_status() == 0
+    pool.close(); model.close()
+
+
+# ---------------------------------------------------------------- pointwise (HSTU-style) attention
+def test_pointwise_attention_fp32_matches_checker():
+    """Config-1 batch and model with attn_kind = pointwise: psi, rank on cache and full inference against the checker."""
+    import dataclasses
+    wl = synth.workload(1)
+    shape = dataclasses.replace(wl.model, attn_kind=1)
+    rng = np.random.default_rng(wl.seed)
+    batch = synth.config1_batch(synth.ZipfIds(shape.vocab, wl.zipf_a), rng)
+    w, model, pool, db = _setup(shape, wl.seed, batch)
+    om = oracle_model(shape, w)
+    pool.preinfer(db)
+    scores = pool.rank(db)
+    full = model.rank_full(db)
+    torch.cuda.synchronize()
+    for i in range(batch.n_users):
+        p, _, _ = batch.user_slices(i)
+        K, V = om.preinfer(p)
+        gK, gV = pool.read_kv(batch.users[i], len(p))
+        assert np.max(np.abs(gK.cpu().numpy().astype(np.float64) - K)) <= TOL_F32
+        assert np.max(np.abs(gV.cpu().numpy().astype(np.float64) - V)) <= TOL_F32
+    want = oracle_scores(om, batch)
+    assert max_abs_err(scores.cpu().numpy(), batch, want) <= TOL_F32
+    assert max_abs_err(full.cpu().numpy(), batch, want) <= TOL_F32
+    # and it is a different model from the softmax one
+    soft = oracle_scores(oracle_model(wl.model, w), batch, users=[0])
+    assert np.max(np.abs(soft[0] - want[0])) > 1e-2
+    assert model.device_status() == 0
+    pool.close(); model.close()
+
+
+POINTWISE = [
+    ([300, 129, 64, 1000], [5, 0, 70, 33], [130, 7, 0, 257]),      # jagged: ragged tiles, empty segments
+    ([1, 63, 65, 128], [0, 1, 0, 130], [1, 0, 129, 3]),
+    ([4096], [64], [200]),                                         # one long user: the key range is split and merged
+]
+
+
+@pytest.mark.parametrize("case", range(len(POINTWISE)))
+def test_pointwise_attention_bf16_matches_checker(case):
+    p, s, c = POINTWISE[case]
+    shape = small_bf16_shape(attn_kind=1)
+    batch = _tiny_batch(shape, 70 + case, p, s, c)
+    w, model, pool, db = _setup(shape, 23, batch)
+    om = oracle_model(shape, w)
+    pool.preinfer(db)
+    scores = pool.rank(db)
+    full = model.rank_full(db)
+    torch.cuda.synchronize()
+    for i in range(batch.n_users):
+        pp, _, _ = batch.user_slices(i)
+        K, V = om.preinfer(pp)
+        gK, gV = pool.read_kv(batch.users[i], len(pp))
+        assert np.max(np.abs(gK.float().cpu().numpy() - K)) <= 5e-2
+        assert np.max(np.abs(gV.float().cpu().numpy() - V)) <= 5e-2
+    want = oracle_scores(om, batch)
+    assert max_abs_err(scores.cpu().numpy(), batch, want) <= TOL_BF16_POINTWISE
+    assert max_abs_err(full.cpu().numpy(), batch, want) <= TOL_BF16_POINTWISE
+    assert np.std(np.concatenate([v for v in want.values() if len(v)])) > 0.3          # scores are not degenerate
     assert model.device_status() == 0
     pool.close(); model.close()
