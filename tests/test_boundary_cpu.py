@@ -42,6 +42,15 @@ def test_shape_validation():
         with pytest.raises(B.RelayGRError):
             B.relaygr_create_host_only(bad)
     assert "d_head" in B.last_error() or "n_layers" in B.last_error() or "positive" in B.last_error()
+    with pytest.raises(B.RelayGRError):                                          # attn_kind is softmax (0) or pointwise (1)
+        B.relaygr_create_host_only(B.ModelCfg(2, 128, 2, 64, 256, B.DTYPE_F32, 64, 10, 1e-5, 2))
+    assert "attn_kind" in B.last_error()
+
+
+def test_both_attention_kinds_are_accepted():
+    for kind in (0, 1):
+        ctx = B.relaygr_create_host_only(B.ModelCfg(2, 128, 2, 64, 256, B.DTYPE_BF16, 64, 10, 1e-5, kind))
+        B.relaygr_destroy(ctx)
 
 
 def test_no_cpu_compute_path():
