@@ -30,6 +30,7 @@ namespace {
 constexpr int kQTile = 128, kKeys = 64, kDh = 64;
 constexpr int kQBytes = kQTile * kDh * 2;           // 16 KB
 constexpr int kKVBytes = kKeys * kDh * 2;           // 8 KB per K or V tile
+constexpr bool kOffload = true;                       // a quarter of the exponentials runs on the FMA pipe (exp2_fma_pipe)
 constexpr int kStagesKV = 4;
 constexpr int kSmemBytes = kQBytes + 2 * kStagesKV * kKVBytes + 1024 + 512;
 constexpr uint32_t kTmemCols = 256;                 // S[2]: 0..127, P[2]: 128..191, O: 192..255
@@ -70,6 +71,31 @@ __device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b)
     asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
     return d;
 }
+// 2^x for a packed pair WITHOUT the XU pipe: x is rounded to the nearest integer n by adding 1.5 * 2^23 (n then sits in
+// the low mantissa bits), a cubic gives 2^(x - n) on [-0.5, 0.5] (relative error 7.5e-5, far below the bf16 rounding of P
+// that follows) and n is added to the exponent field as an integer.  x is clamped to [-126, 126] first: below that the
+// result is ~1e-38 instead of 0 (a masked key's -inf included: its weight stays negligible), above it the row-sum check
+// of the caller fails and the block is redone against a true maximum.
+__device__ __forceinline__ void exp2_fma_pipe(uint64_t x2, float &p0, float &p1)
+{
+    float x0, x1;
+    unpack2(x2, x0, x1);
+    x0 = fminf(fmaxf(x0, -126.f), 126.f);
+    x1 = fminf(fmaxf(x1, -126.f), 126.f);
+    const uint64_t xc = pack2(x0, x1);
+    const uint64_t r2 = add2(xc, pack2(12582912.f, 12582912.f));
+    const uint64_t n2 = add2(r2, pack2(-12582912.f, -12582912.f));
+    const uint64_t f2 = fma2(n2, pack2(-1.f, -1.f), xc);
+    uint64_t q2 = fma2(pack2(0.0551716685f, 0.0551716685f), f2, pack2(0.2426111251f, 0.2426111251f));
+    q2 = fma2(q2, f2, pack2(0.6932609677f, 0.6932609677f));
+    q2 = fma2(q2, f2, pack2(0.9999280572f, 0.9999280572f));
+    float r0, r1, q0, q1;
+    unpack2(r2, r0, r1);
+    unpack2(q2, q0, q1);
+    p0 = __uint_as_float(__float_as_uint(q0) + (__float_as_uint(r0) << 23));
+    p1 = __uint_as_float(__float_as_uint(q1) + (__float_as_uint(r1) << 23));
+}
+
 __device__ __forceinline__ float max3(float a, float b, float c)
 {
     float d;
@@ -273,30 +299,35 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             // are first taken against the running maximum as it stood before this block; only if the row sum shows that
             // some p may have exceeded 2^8 (or the row has no maximum yet) is the block maximum computed, the running
             // maximum raised, O rescaled and the block redone.  No maximum is on the fast path.
+            // Every fourth pair takes its exponentials on the FMA pipe instead (exp2_fma_pipe): the XU pipe is what the two
+            // CTAs of an SM compete for (measured: 5-7 % off a rank launch; an eighth or three eighths gain less).  (A compile-time pattern: a run-time switch between the two forms inside
+            // the unrolled block cost more than the off-loading gains.)
             auto exp_block = [&](float mc) {
                 const uint64_t c2 = pack2(c, c), nmc2 = pack2(-mc, -mc);
                 uint64_t ra = pack2(0.f, 0.f), rb = ra;
                 uint32_t pk[16];
 #pragma unroll
-                for (int i = 0; i < 16; i += 2) {
-                    float x0, x1, x2, x3;
-                    unpack2(fma2(pack2(__uint_as_float(s0[2 * i]), __uint_as_float(s0[2 * i + 1])), c2, nmc2), x0, x1);
-                    unpack2(fma2(pack2(__uint_as_float(s0[2 * i + 2]), __uint_as_float(s0[2 * i + 3])), c2, nmc2), x2, x3);
-                    const float p0 = ex2(x0), p1 = ex2(x1), p2 = ex2(x2), p3 = ex2(x3);
-                    ra = add2(ra, pack2(p0, p1)); rb = add2(rb, pack2(p2, p3));
-                    pk[i] = tc::pack_bf16(p0, p1); pk[i + 1] = tc::pack_bf16(p2, p3);
-                }
-                tc::tmem_st16(lane_addr + kColP + b * (kKeys / 2), pk);
+                for (int half = 0; half < 2; ++half) {
 #pragma unroll
-                for (int i = 0; i < 16; i += 2) {
-                    float x0, x1, x2, x3;
-                    unpack2(fma2(pack2(__uint_as_float(s1[2 * i]), __uint_as_float(s1[2 * i + 1])), c2, nmc2), x0, x1);
-                    unpack2(fma2(pack2(__uint_as_float(s1[2 * i + 2]), __uint_as_float(s1[2 * i + 3])), c2, nmc2), x2, x3);
-                    const float p0 = ex2(x0), p1 = ex2(x1), p2 = ex2(x2), p3 = ex2(x3);
-                    ra = add2(ra, pack2(p0, p1)); rb = add2(rb, pack2(p2, p3));
-                    pk[i] = tc::pack_bf16(p0, p1); pk[i + 1] = tc::pack_bf16(p2, p3);
+                    for (int i = 0; i < 16; i += 2) {
+                        const uint32_t a0 = half == 0 ? s0[2 * i] : s1[2 * i], a1 = half == 0 ? s0[2 * i + 1] : s1[2 * i + 1];
+                        const uint32_t a2 = half == 0 ? s0[2 * i + 2] : s1[2 * i + 2], a3 = half == 0 ? s0[2 * i + 3] : s1[2 * i + 3];
+                        const uint64_t xa = fma2(pack2(__uint_as_float(a0), __uint_as_float(a1)), c2, nmc2);
+                        const uint64_t xb = fma2(pack2(__uint_as_float(a2), __uint_as_float(a3)), c2, nmc2);
+                        float p0, p1, p2, p3, x0, x1, x2, x3;
+                        unpack2(xb, x2, x3);
+                        p2 = ex2(x2); p3 = ex2(x3);
+                        if (kOffload && (i & 2) != 0) {
+                            exp2_fma_pipe(xa, p0, p1);
+                        } else {
+                            unpack2(xa, x0, x1);
+                            p0 = ex2(x0); p1 = ex2(x1);
+                        }
+                        ra = add2(ra, pack2(p0, p1)); rb = add2(rb, pack2(p2, p3));
+                        pk[i] = tc::pack_bf16(p0, p1); pk[i + 1] = tc::pack_bf16(p2, p3);
+                    }
+                    tc::tmem_st16(lane_addr + kColP + b * (kKeys / 2) + 16 * half, pk);
                 }
-                tc::tmem_st16(lane_addr + kColP + b * (kKeys / 2) + 16, pk);
                 float r0, r1;
                 unpack2(add2(ra, rb), r0, r1);
                 return r0 + r1;
