@@ -30,7 +30,10 @@ namespace {
 constexpr int kQTile = 128, kKeys = 64, kDh = 64;
 constexpr int kQBytes = kQTile * kDh * 2;           // 16 KB
 constexpr int kKVBytes = kKeys * kDh * 2;           // 8 KB per K or V tile
-constexpr bool kOffload = true;                       // a quarter of the exponentials runs on the FMA pipe (exp2_fma_pipe)
+#ifndef RELAYGR_ATTN_OFFLOAD
+#define RELAYGR_ATTN_OFFLOAD 1
+#endif
+constexpr bool kOffload = RELAYGR_ATTN_OFFLOAD != 0;                       // a quarter of the exponentials runs on the FMA pipe (exp2_fma_pipe)
 constexpr int kStagesKV = 4;
 constexpr int kSmemBytes = kQBytes + 2 * kStagesKV * kKVBytes + 1024 + 512;
 constexpr uint32_t kTmemCols = 256;                 // S[2]: 0..127, P[2]: 128..191, O: 192..255
