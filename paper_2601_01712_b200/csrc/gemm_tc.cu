@@ -360,7 +360,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 }
             }
         }
-        if (lane == 0) tc::bulk_wait<0>();                  // this warp's stores have been performed
+        if (lane == 0) tc::bulk_wait_read<0>();             // the patch has been read; the grid's completion covers the global writes
     }
     tc::tc_fence_before();
     __syncthreads();
