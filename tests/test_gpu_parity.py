@@ -439,3 +439,23 @@ def test_pointwise_attention_bf16_matches_checker(case):
     assert np.std(np.concatenate([v for v in want.values() if len(v)])) > 0.3          # scores are not degenerate
     assert model.device_status() == 0
     pool.close(); model.close()
+
+
+# ---------------------------------------------------------------- feed-forward widths around the fused kernel's limits
+@pytest.mark.parametrize("ff", [128, 2048, 2304])
+def test_feed_forward_widths_d256(ff):
+    """d_model = 256 with one hidden chunk, with the widest fused feed-forward (2048) and just past it (2304: LayerNorm and
+    two GEMM launches instead), on a jagged batch with a ragged last tile."""
+    shape = small_bf16_shape(ff=ff)
+    batch = _tiny_batch(shape, 90 + ff, [200, 70, 333], [3, 40, 0], [65, 0, 131])
+    w, model, pool, db = _setup(shape, 29, batch)
+    om = oracle_model(shape, w)
+    pool.preinfer(db)
+    scores = pool.rank(db)
+    full = model.rank_full(db)
+    torch.cuda.synchronize()
+    want = oracle_scores(om, batch)
+    assert max_abs_err(scores.cpu().numpy(), batch, want) <= TOL_BF16
+    assert max_abs_err(full.cpu().numpy(), batch, want) <= TOL_BF16
+    assert model.device_status() == 0
+    pool.close(); model.close()
