@@ -1,19 +1,24 @@
 // bf16 GEMM on the 5th-generation tensor cores: C[m, n] = sum_k A[m, k] W[n, k] with fp32
 // accumulators in TMEM.  The K extents of this model are short (d_model or d_ff), so a tile's
-// mainloop is a handful of MMAs and the epilogue - reading 128 x BN accumulators back and
-// moving them to global memory - is the longer half.  The kernel is therefore persistent
-// (one CTA per SM walks a list of 128 x BN output tiles) with two accumulators in TMEM, so
+// mainloop is a handful of MMAs and the epilogue - reading the accumulators back and moving
+// them to global memory - weighs as much.  The kernel is therefore persistent (one CTA, or one
+// CTA pair, per SM or SM pair walks a list of output tiles) with two accumulators in TMEM, so
 // that the epilogue of one tile runs under the TMA loads and MMAs of the next, and the
 // epilogue hands its output to the TMA unit: a warp stages 32 rows x 128 bytes in shared
 // memory (128-byte swizzle, conflict-free) and one lane issues a bulk tensor store - or, for
 // the residual stream, a bulk fp32 add-reduction (x += tile, performed in L2: the residual
-// never travels to the SM).  Only K/V rows that go straight into a user's pages are written
-// with plain stores (their destination is a page-table walk per row).
+// never travels to the SM).  K/V rows of a pre-infer call go straight into the users' pages:
+// with one bulk tensor store where a warp's 32 rows are 32 consecutive slots of one page,
+// with plain stores after a page-table walk per row otherwise.
 //
-// Warp roles (320 threads): warp 0 = TMA producer (128 x 64 tiles of A and W, 128-byte
-// swizzle, 3-4-stage ring), warp 1 = TMEM owner + MMA issuer (tcgen05.mma M128 N = BN K16),
-// warps 2-9 = epilogue: warp w reads TMEM lanes 32 (w % 4) .. +31 (its hardware quadrant),
-// columns (BN / 2) ((w - 2) / 4) .. + BN / 2 - 1, 64 at a time, applies bias / SiLU in the
+// Two shapes (Cfg below): single CTAs with 128 x 128 tiles, and CTA pairs (a cluster of two,
+// tcgen05 cta_group::2) with 256 x 256 tiles, where each CTA loads its 128 rows of A and half
+// of W and the even CTA issues the MMAs for both.
+//
+// Warp roles (320 threads per CTA): warp 0 = TMA producer (128 x 64 tiles of A and W, 128-byte
+// swizzle, five-stage ring), warp 1 = TMEM owner + MMA issuer (tcgen05.mma K16), warps 2-9 =
+// epilogue: warp w reads TMEM lanes 32 (w % 4) .. +31 (its hardware quadrant), columns
+// (BN / 2) ((w - 2) / 4) .. + BN / 2 - 1, 64 at a time, applies bias / SiLU in the
 // row-per-thread layout tcgen05.ld delivers and stages the result for the store.
 #include "kernels.cuh"
 #include "tc_common.cuh"

@@ -330,7 +330,7 @@ def test_two_model_slots_share_one_pool():
 # ---------------------------------------------------------------- other widths, edge shapes
 @pytest.mark.parametrize("d,heads,ff,layers", [(128, 2, 512, 3), (384, 6, 1536, 2), (1024, 16, 4096, 2)])
 def test_other_model_widths_match_checker(d, heads, ff, layers):
-    """Widths that take the other tile shapes of the GEMM (N not a multiple of 256; the 256-wide long-K tile) and 2 / 6 / 16 heads."""
+    """Widths that take both GEMM shapes (single CTAs where N is not a multiple of 256, CTA pairs elsewhere) and 2 / 6 / 16 heads."""
     shape = small_bf16_shape(vocab=3000, layers=layers, d=d, heads=heads, ff=ff)
     batch = _tiny_batch(shape, 50 + d, [333, 64, 129], [7, 0, 65], [70, 130, 1])
     w, model, pool, db = _setup(shape, 27, batch)
