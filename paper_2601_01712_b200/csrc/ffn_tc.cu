@@ -33,7 +33,9 @@ constexpr int kStageBytes = 32 * 1024, kStages = 4;
 constexpr int kOffW = kABytes;
 constexpr int kOffB1 = kOffW + kStages * kStageBytes;
 constexpr int kOffB2 = kOffB1 + kMaxF * 4;
-constexpr int kOffBars = kOffB2 + kD * 4;
+constexpr int kOffG = kOffB2 + kD * 4;               // LayerNorm gain and offset, out-proj bias (kProj): 3 x 256 floats
+constexpr int kOffStat = kOffG + 3 * kD * 4;         // partial row statistics exchanged between the two warps of a row: 2 x 2 x 128 floats
+constexpr int kOffBars = kOffStat + 2 * 2 * kRows * 4;
 constexpr int kSmemBytes = kOffBars + 256 + 1024;
 static_assert(kSmemBytes <= 227 * 1024, "shared memory budget");
 constexpr uint32_t kTmemCols = 512, kColO = 0, kColS = 256;      // S buffer i at kColS + 128 i; H(c) in the first 64 columns of S(c)'s buffer
@@ -44,6 +46,7 @@ struct Bars {
     uint64_t s_full[2];                               // S(c) complete in buffer c & 1
     uint64_t h_full[2];                               // H(c) in TMEM (256 arrivals)
     uint64_t o_full;
+    uint64_t att_full, o1_full, x_full[4], x_done;    // kProj: attention tile landed / att Wo^T complete / x rows landed / x consumed
     uint32_t tmem_slot;
     int abort_flag;
 };
@@ -69,15 +72,22 @@ __device__ __forceinline__ uint4 *patch_chunk(uint8_t *patch, int r, int j)
     return reinterpret_cast<uint4 *>(patch + r * 128 + ((j ^ (r & 7)) << 4));
 }
 
+// kProj: the output projection of the attention block runs first, in the same kernel: O starts as att Wo^T, LayerNorm is
+// taken of x + O + bo (the block's mid-point, never written), and the feed-forward MMAs accumulate on top, so that the
+// final add-reduction adds (att Wo^T + bo) + (feed-forward + b2) to x in one go.
+template <bool kProj>
 __global__ void __launch_bounds__(kThreads, 1)
 ffn_fused_kernel(const __grid_constant__ CUtensorMap tmW1, const __grid_constant__ CUtensorMap tmW2, const __grid_constant__ CUtensorMap tmX,
+                 const __grid_constant__ CUtensorMap tmAtt, const __grid_constant__ CUtensorMap tmWo,
                  const float *__restrict__ x, const float *__restrict__ g, const float *__restrict__ b, const float *__restrict__ b1,
-                 const float *__restrict__ b2, int64_t M, int F, float eps, int *err)
+                 const float *__restrict__ b2, const float *__restrict__ bo, int64_t M, int F, float eps, int *err)
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t *sA = smem, *sW = smem + kOffW;
     float *b1s = reinterpret_cast<float *>(smem + kOffB1), *b2s = reinterpret_cast<float *>(smem + kOffB2);
+    float *gs = reinterpret_cast<float *>(smem + kOffG), *bs = gs + kD, *bos = bs + kD;
+    float *stat = reinterpret_cast<float *>(smem + kOffStat);
     Bars *bars = reinterpret_cast<Bars *>(smem + kOffBars);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -90,6 +100,8 @@ ffn_fused_kernel(const __grid_constant__ CUtensorMap tmW1, const __grid_constant
         for (int s = 0; s < kStages; ++s) { tc::mbar_init(&bars->w_full[s], 1); tc::mbar_init(&bars->w_empty[s], 1); }
         for (int i = 0; i < 2; ++i) { tc::mbar_init(&bars->s_full[i], 1); tc::mbar_init(&bars->h_full[i], kEpiThreads); }
         tc::mbar_init(&bars->o_full, 1);
+        tc::mbar_init(&bars->att_full, 1); tc::mbar_init(&bars->o1_full, 1); tc::mbar_init(&bars->x_done, kEpiThreads);
+        for (int i = 0; i < 4; ++i) tc::mbar_init(&bars->x_full[i], 1);
         tc::fence_mbar_init();
         tc::tma_prefetch_desc(&tmW1); tc::tma_prefetch_desc(&tmW2); tc::tma_prefetch_desc(&tmX);
     }
@@ -99,7 +111,10 @@ ffn_fused_kernel(const __grid_constant__ CUtensorMap tmW1, const __grid_constant
     }
     if (warp >= 2) {                                  // the biases are parameters: not written by earlier kernels
         for (int i = threadIdx.x - 64; i < F; i += kEpiThreads) b1s[i] = b1 ? b1[i] : 0.f;
-        for (int i = threadIdx.x - 64; i < kD; i += kEpiThreads) b2s[i] = b2 ? b2[i] : 0.f;
+        for (int i = threadIdx.x - 64; i < kD; i += kEpiThreads) {
+            b2s[i] = (b2 ? b2[i] : 0.f) + (kProj && bo ? bo[i] : 0.f);      // what the final add-reduction adds beside O
+            if (kProj) { gs[i] = g[i]; bs[i] = b[i]; bos[i] = bo ? bo[i] : 0.f; }
+        }
     }
     grid_launch_dependents();
     grid_dependency_wait();                           // from here on: data of earlier kernels
@@ -132,6 +147,26 @@ ffn_fused_kernel(const __grid_constant__ CUtensorMap tmW1, const __grid_constant
                 }
                 ++it;
             };
+            if (kProj) {
+                // the attention tile (A of the projection) where the normalised tile will go, Wo through the ring, then - once
+                // the projection MMAs have read both - this CTA's rows of x into the ring's memory as 32 x 32 fp32 patches
+                tc::mbar_expect_tx(&bars->att_full, kABytes);
+                for (int kb = 0; kb < 4; ++kb) tc::tma_load_2d(sA + kb * kKBlock, &tmAtt, kb * 64, (int)m0, &bars->att_full);
+                for (int kb = 0; kb < 4 && ok; ++kb, ++it) {
+                    const int s = it % kStages;
+                    ok = tc::mbar_wait(&bars->w_empty[s], ((it / kStages) & 1) ^ 1, err);
+                    if (!ok) break;
+                    tc::mbar_expect_tx(&bars->w_full[s], kStageBytes);
+                    tc::tma_load_2d(sW + s * kStageBytes, &tmWo, kb * 64, 0, &bars->w_full[s]);
+                }
+                if (ok) ok = tc::mbar_wait(&bars->o1_full, 0, err);
+                for (int rg = 0; rg < 4 && ok; ++rg) {
+                    tc::mbar_expect_tx(&bars->x_full[rg], kStageBytes);
+                    for (int cg = 0; cg < 8; ++cg)
+                        tc::tma_load_2d(sW + (rg * 8 + cg) * 4096, &tmX, cg * 32, (int)(m0 + rg * 32), &bars->x_full[rg]);
+                }
+                if (ok) ok = tc::mbar_wait(&bars->x_done, 0, err);          // the LayerNorm has taken x: the ring is free for weights
+            }
             load(false, 0, 0); load(false, 0, 1);
             if (n_chunks > 1) { load(false, 1, 0); load(false, 1, 1); }
             for (int c = 0; c < n_chunks; ++c) {
@@ -144,9 +179,27 @@ ffn_fused_kernel(const __grid_constant__ CUtensorMap tmW1, const __grid_constant
         constexpr uint32_t idesc_s = tc::make_idesc(kRows, kChunk, 0, 0);      // A and W1 both K-major
         constexpr uint32_t idesc_o = tc::make_idesc(kRows, kD, 0, 0);          // H from TMEM, W2 K-major
         uint32_t it = 0;
-        bool ok = tc::mbar_wait(&bars->a_ready, 0, err);
-        tc::tc_fence_after();
+        bool ok = true;
         const uint32_t a0 = tc::smem_u32(sA);
+        if (kProj) {                                  // O = att Wo^T: four K blocks, M128 N256
+            ok = tc::mbar_wait(&bars->att_full, 0, err);
+            for (int kb = 0; kb < 4 && ok; ++kb, ++it) {
+                const int s = it % kStages;
+                ok = tc::mbar_wait(&bars->w_full[s], (it / kStages) & 1, err);
+                if (!ok) break;
+                tc::tc_fence_after();
+                const uint64_t adesc = tc::smem_desc_sw128(a0 + kb * kKBlock), bdesc = tc::smem_desc_sw128(tc::smem_u32(sW + s * kStageBytes));
+                if (tc::elect_one()) {
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) tc::mma_ss(tmem_base + kColO, adesc + 2 * k, bdesc + 2 * k, idesc_o, (kb | k) != 0);
+                    tc::mma_commit(&bars->w_empty[s]);
+                    if (kb == 3) tc::mma_commit(&bars->o1_full);
+                }
+                __syncwarp();
+            }
+        }
+        if (ok) ok = tc::mbar_wait(&bars->a_ready, 0, err);
+        tc::tc_fence_after();
         auto issue_s = [&](int c) {                   // S(c) = A W1c^T: two stages, each two K blocks of 64
             const uint32_t scol = kColS + (c & 1) * kChunk;
             for (int half = 0; half < 2 && ok; ++half, ++it) {
@@ -179,7 +232,7 @@ ffn_fused_kernel(const __grid_constant__ CUtensorMap tmW1, const __grid_constant
                 if (tc::elect_one()) {
 #pragma unroll
                     for (int k = 0; k < 4; ++k)      // 16 hidden units per instruction: 8 TMEM columns of H, 32 bytes of every W2 row
-                        tc::mma_ts(tmem_base + kColO, tmem_base + hcol + half * 64 + k * 8, bdesc + 2 * k, idesc_o, (c | half | k) != 0);
+                        tc::mma_ts(tmem_base + kColO, tmem_base + hcol + half * 64 + k * 8, bdesc + 2 * k, idesc_o, kProj || (c | half | k) != 0);
                     tc::mma_commit(&bars->w_empty[s]);
                     if (half == 1 && c == n_chunks - 1) tc::mma_commit(&bars->o_full);
                 }
@@ -201,7 +254,62 @@ ffn_fused_kernel(const __grid_constant__ CUtensorMap tmW1, const __grid_constant
         const int ew = warp - 2, quad = warp & 3, ch = ew >> 2;
         const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
         bool ok = true;
-        {
+        if (kProj) {
+            // mid = x + att Wo^T + bo, one row per thread (the layout TMEM delivers), this warp's 128 columns of it in registers;
+            // a = LN(mid) into the tile the attention rows came in.  The row statistics need both column halves: the two warps
+            // of a row exchange partial sums through shared memory.
+            const int rr = quad * 32 + lane;
+            ok = __all_sync(0xffffffffu, tc::mbar_wait(&bars->o1_full, 0, err));
+            if (ok) ok = __all_sync(0xffffffffu, tc::mbar_wait(&bars->x_full[quad], 0, err));
+            tc::tc_fence_after();
+            float xp[128];
+            float psum = 0.f;
+#pragma unroll
+            for (int gi = 0; gi < 4; ++gi) {
+                const int cc = ch * 128 + gi * 32;
+                uint32_t r[32];
+                tc::tmem_ld32(lane_addr + kColO + cc, r);
+                tc::tmem_ld_wait();
+                const uint8_t *patch = sW + (quad * 8 + ch * 4 + gi) * 4096;
+#pragma unroll
+                for (int jj = 0; jj < 8; ++jj) {
+                    const uint4 xv = *patch_chunk(const_cast<uint8_t *>(patch), lane, jj);
+                    const float4 q = *reinterpret_cast<const float4 *>(bos + cc + 4 * jj);
+                    xp[gi * 32 + 4 * jj] = __uint_as_float(r[4 * jj]) + __uint_as_float(xv.x) + q.x;
+                    xp[gi * 32 + 4 * jj + 1] = __uint_as_float(r[4 * jj + 1]) + __uint_as_float(xv.y) + q.y;
+                    xp[gi * 32 + 4 * jj + 2] = __uint_as_float(r[4 * jj + 2]) + __uint_as_float(xv.z) + q.z;
+                    xp[gi * 32 + 4 * jj + 3] = __uint_as_float(r[4 * jj + 3]) + __uint_as_float(xv.w) + q.w;
+                    psum += (xp[gi * 32 + 4 * jj] + xp[gi * 32 + 4 * jj + 1]) + (xp[gi * 32 + 4 * jj + 2] + xp[gi * 32 + 4 * jj + 3]);
+                }
+            }
+            stat[ch * kRows + rr] = psum;
+            asm volatile("bar.sync 1, 256;" ::: "memory");
+            const float mean = (stat[rr] + stat[kRows + rr]) * (1.f / kD);
+            float pvar = 0.f;
+#pragma unroll
+            for (int i = 0; i < 128; ++i) { const float dlt = xp[i] - mean; pvar = fmaf(dlt, dlt, pvar); }
+            stat[(2 + ch) * kRows + rr] = pvar;
+            asm volatile("bar.sync 1, 256;" ::: "memory");
+            const float rstd = rsqrtf((stat[2 * kRows + rr] + stat[3 * kRows + rr]) * (1.f / kD) + eps);
+#pragma unroll
+            for (int q16 = 0; q16 < 16; ++q16) {
+                const int c = ch * 128 + q16 * 8;
+                const float4 ga = *reinterpret_cast<const float4 *>(gs + c), gb = *reinterpret_cast<const float4 *>(gs + c + 4);
+                const float4 ba = *reinterpret_cast<const float4 *>(bs + c), bb2 = *reinterpret_cast<const float4 *>(bs + c + 4);
+                const float *v = xp + q16 * 8;
+                uint4 o;
+                o.x = tc::pack_bf16((v[0] - mean) * rstd * ga.x + ba.x, (v[1] - mean) * rstd * ga.y + ba.y);
+                o.y = tc::pack_bf16((v[2] - mean) * rstd * ga.z + ba.z, (v[3] - mean) * rstd * ga.w + ba.w);
+                o.z = tc::pack_bf16((v[4] - mean) * rstd * gb.x + bb2.x, (v[5] - mean) * rstd * gb.y + bb2.y);
+                o.w = tc::pack_bf16((v[6] - mean) * rstd * gb.z + bb2.z, (v[7] - mean) * rstd * gb.w + bb2.w);
+                const int kb = c >> 6, j = (c & 63) >> 3;
+                *reinterpret_cast<uint4 *>(sA + kb * kKBlock + rr * 128 + ((j ^ (rr & 7)) << 4)) = o;
+            }
+            tc::fence_proxy_async();                  // generic-proxy writes of the tile before the tensor core reads it
+            tc::tc_fence_before();
+            tc::mbar_arrive(&bars->x_done);
+            tc::mbar_arrive(&bars->a_ready);
+        } else {
             // a[r, :] = LN(x[r, :]) for 16 rows per warp, all their loads in flight at once: lane l holds columns 8l .. 8l+7,
             // i.e. the 16-byte chunk (l & 7) of K block (l >> 3), stored with the 128-byte swizzle the MMA descriptor expects
             const float4 g0 = *reinterpret_cast<const float4 *>(g + 8 * lane), g1 = *reinterpret_cast<const float4 *>(g + 8 * lane + 4);
@@ -306,19 +414,24 @@ ffn_fused_kernel(const __grid_constant__ CUtensorMap tmW1, const __grid_constant
 bool ffn_fused_supported(int d_model, int d_ff) { return d_model == kD && d_ff % kChunk == 0 && d_ff >= kChunk && d_ff <= kMaxF; }
 
 cudaError_t launch_ffn_fused(const CUtensorMap &tmW1, const CUtensorMap &tmW2, const CUtensorMap &tmX, const float *x, const float *g,
-                             const float *b, const float *b1, const float *b2, int64_t M, int d_ff, float eps, int *err,
-                             cudaStream_t stream, int64_t *launches)
+                             const float *b, const float *b1, const float *b2, const CUtensorMap *tmAtt, const CUtensorMap *tmWo,
+                             const float *bo, int64_t M, int d_ff, float eps, int *err, cudaStream_t stream, int64_t *launches)
 {
     if (M == 0) return cudaSuccess;
     static bool attr_set = false;
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(ffn_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        cudaError_t e = cudaFuncSetAttribute(ffn_fused_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(ffn_fused_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
     *launches += 1;
-    return launch_dependent(ffn_fused_kernel, dim3((unsigned)((M + kRows - 1) / kRows)), dim3(kThreads), (size_t)kSmemBytes, stream, 1, tmW1, tmW2,
-                            tmX, x, g, b, b1, b2, M, d_ff, eps, err);
+    const dim3 grid((unsigned)((M + kRows - 1) / kRows));
+    if (tmAtt && tmWo)
+        return launch_dependent(ffn_fused_kernel<true>, grid, dim3(kThreads), (size_t)kSmemBytes, stream, 1, tmW1, tmW2, tmX, *tmAtt, *tmWo, x, g,
+                                b, b1, b2, bo, M, d_ff, eps, err);
+    return launch_dependent(ffn_fused_kernel<false>, grid, dim3(kThreads), (size_t)kSmemBytes, stream, 1, tmW1, tmW2, tmX, tmX, tmX, x, g, b, b1,
+                            b2, bo, M, d_ff, eps, err);
 }
 
 }  // namespace relaygr

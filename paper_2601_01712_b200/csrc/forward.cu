@@ -82,8 +82,10 @@ int Forward::init_device(int dev, std::string &err)
             rc |= make_tmap_2d_bf16(&wmaps[(size_t)l].wo, (const __nv_bfloat16 *)w.w_o + (size_t)l * d * d, d, d, d, (uint32_t)kGemmWeightBoxRows, 64);
             rc |= make_tmap_2d_bf16(&wmaps[(size_t)l].w1, (const __nv_bfloat16 *)w.w1 + (size_t)l * F * d, F, d, d, (uint32_t)kGemmWeightBoxRows, 64);
             rc |= make_tmap_2d_bf16(&wmaps[(size_t)l].w2, (const __nv_bfloat16 *)w.w2 + (size_t)l * d * F, d, F, F, (uint32_t)kGemmWeightBoxRows, 64);
-            if (ffn_fused_supported((int)d, (int)F))
+            if (ffn_fused_supported((int)d, (int)F)) {
                 rc |= make_tmap_2d_bf16(&wmaps[(size_t)l].w2_wide, (const __nv_bfloat16 *)w.w2 + (size_t)l * d * F, d, F, F, 256, 64);
+                rc |= make_tmap_2d_bf16(&wmaps[(size_t)l].wo_wide, (const __nv_bfloat16 *)w.w_o + (size_t)l * d * d, d, d, d, 256, 64);
+            }
             if (rc != 0) { err = "tensor-map encoding of the weights failed (pointers must be 16-byte aligned)"; return RELAYGR_E_CUDA; }
         }
     }
@@ -377,21 +379,21 @@ int Forward::run_t(const CallDesc &call, float *scores, cudaStream_t stream, std
         }
         if (!ck("attention")) return RELAYGR_E_CUDA;
 
+        if (kTensor && ffn_fused_supported((int)d, (int)F)) {
+            // output projection + residual, LayerNorm 2, both feed-forward GEMMs, SiLU and the second residual add in one kernel
+            cudaEvent_t pe = prof_begin(stream);
+            e = launch_ffn_fused(lm->w1, lm->w2_wide, om_x.o[0], x, w.ln2_g + (size_t)l * d, w.ln2_b + (size_t)l * d,
+                                 w.b1 ? w.b1 + (size_t)l * F : nullptr, w.b2 ? w.b2 + (size_t)l * d : nullptr, &tm_att, &lm->wo_wide,
+                                 w.b_o ? w.b_o + (size_t)l * d : nullptr, R, (int)F, cfg.ln_eps, d_status, stream, &launches);
+            prof_end(KC_GEMM, pe, stream);
+            if (!ck("output projection + feed-forward")) return RELAYGR_E_CUDA;
+            continue;
+        }
         Epilogue eo{};
         eo.mode = EPI_RESID; eo.bias = w.b_o ? w.b_o + (size_t)l * d : nullptr; eo.resid = x; eo.out_f32 = x;
         e = gemm(att, tm_att, (const T *)w.w_o + (size_t)l * d * d, lm ? &lm->wo : nullptr, om_x, d, d, eo);
         if (!ck("output projection")) return RELAYGR_E_CUDA;
 
-        if (kTensor && ffn_fused_supported((int)d, (int)F)) {
-            // LayerNorm 2, both feed-forward GEMMs, SiLU and the residual add in one kernel
-            cudaEvent_t pe = prof_begin(stream);
-            e = launch_ffn_fused(lm->w1, lm->w2_wide, om_x.o[0], x, w.ln2_g + (size_t)l * d, w.ln2_b + (size_t)l * d,
-                                 w.b1 ? w.b1 + (size_t)l * F : nullptr, w.b2 ? w.b2 + (size_t)l * d : nullptr, R, (int)F, cfg.ln_eps, d_status,
-                                 stream, &launches);
-            prof_end(KC_GEMM, pe, stream);
-            if (!ck("feed-forward")) return RELAYGR_E_CUDA;
-            continue;
-        }
         e = layernorm(w.ln2_g + (size_t)l * d, w.ln2_b + (size_t)l * d);
         if (!ck("LayerNorm 2")) return RELAYGR_E_CUDA;
 

@@ -43,7 +43,7 @@ struct Forward {
     int n_sms = 148;
 
     // tensor maps of the weights (bf16 model), one set per layer
-    struct LayerMaps { CUtensorMap qkv, kv, wo, w1, w2, w2_wide; };      // w2_wide: W2 in boxes of 256 rows (fused feed-forward)
+    struct LayerMaps { CUtensorMap qkv, kv, wo, w1, w2, w2_wide, wo_wide; };      // *_wide: boxes of 256 rows (fused out-proj + feed-forward)
     std::vector<LayerMaps> wmaps;
 
     // pinned staging ring for the per-call metadata

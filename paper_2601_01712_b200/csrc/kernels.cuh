@@ -95,11 +95,15 @@ cudaError_t launch_gemm_tc(const CUtensorMap &tmA, const CUtensorMap &tmB, const
 // ffn_fused_supported() accepts (d_model = 256, d_ff a multiple of 128 up to 2048): LayerNorm, both GEMMs, SiLU and the
 // residual add without a round trip of the normalised or hidden activations through global memory.  tmW1: W1 [d_ff, 256]
 // in boxes of 128 rows x 64 columns; tmW2: W2 [256, d_ff] in boxes of 256 rows x 64 columns; tmX: the fp32 residual stream
-// [M, 256] in boxes of 32 rows x 32 columns (the target of the add-reduction); all with the 128-byte swizzle.
+// [M, 256] in boxes of 32 rows x 32 columns (read by the LayerNorm of the projection form, target of the add-reduction);
+// all with the 128-byte swizzle.
+// With tmAtt / tmWo (both or neither) the attention block's output projection runs first in the same kernel:
+// mid = x + att Wo^T + bo, x <- mid + W2 SiLU(W1 LN(mid) + b1) + b2.  tmAtt: att [M, 256] bf16 in boxes of 128 rows x 64
+// columns; tmWo: Wo [256, 256] in boxes of 256 rows x 64 columns.
 bool ffn_fused_supported(int d_model, int d_ff);
 cudaError_t launch_ffn_fused(const CUtensorMap &tmW1, const CUtensorMap &tmW2, const CUtensorMap &tmX, const float *x, const float *g,
-                             const float *b, const float *b1, const float *b2, int64_t M, int d_ff, float eps, int *err,
-                             cudaStream_t stream, int64_t *launches);
+                             const float *b, const float *b1, const float *b2, const CUtensorMap *tmAtt, const CUtensorMap *tmWo,
+                             const float *bo, int64_t M, int d_ff, float eps, int *err, cudaStream_t stream, int64_t *launches);
 
 // Flash-style attention on tcgen05 (d_head = 64) over the work items, then the merge of split items.  attn_kind: ATTN_SOFTMAX, or
 // ATTN_POINTWISE (weights SiLU(q.k / sqrt(d_h)) divided by the number of visible keys).
