@@ -31,7 +31,7 @@ WORKLOAD = "config2: 4 layers, d_model 256, 4 heads x 64, FFN 1024, bf16; 32 use
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of this workload's rank step, from the ncu captures
 # summarised under profiles/ (None = no capture of the kernel as it stands).
-DRAM_TRAFFIC_BYTES = {"attention": 120.0e6, "gemm": 19.4e6}      # gemm: mean of QKV, out-proj and the fused feed-forward of a layer
+DRAM_TRAFFIC_BYTES = {"attention": 120.0e6, "gemm": 19.7e6}      # gemm: mean of QKV (9.9 MB) and the fused out-proj + feed-forward kernel (29.6 MB)
 
 
 def load_peaks():
@@ -297,7 +297,7 @@ def main():
     # algorithmic FLOPs of the two tensor-core kernel classes over one rank step (dead last-layer work excluded)
     attn_flops_step = workloads.batch_flops(shape, b0, "rank") - workloads.batch_linear_flops(shape, b0, "rank")
     class_flops = {"attention": attn_flops_step, "gemm": workloads.batch_linear_flops(shape, b0, "rank")}
-    class_name = {"attention": "attention_tc_kernel (rank on cache)", "gemm": "gemm_tc_kernel + ffn_fused_kernel (QKV, out-proj, feed-forward of the rank step)"}
+    class_name = {"attention": "attention_tc_kernel (rank on cache)", "gemm": "gemm_tc_kernel + ffn_fused_kernel (QKV; out-proj + feed-forward of the rank step)"}
     rooflines = {}
     for cls in ("attention", "gemm"):
         n_launch = max(1, prof[cls + "_launches"])
