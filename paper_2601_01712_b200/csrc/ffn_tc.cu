@@ -283,13 +283,13 @@ ffn_fused_kernel(const __grid_constant__ CUtensorMap tmW1, const __grid_constant
                 }
             }
             stat[ch * kRows + rr] = psum;
-            asm volatile("bar.sync 1, 256;" ::: "memory");
+            asm volatile("bar.sync %0, 64;" ::"r"(1 + quad) : "memory");      // the two warps that share these 32 rows
             const float mean = (stat[rr] + stat[kRows + rr]) * (1.f / kD);
             float pvar = 0.f;
 #pragma unroll
             for (int i = 0; i < 128; ++i) { const float dlt = xp[i] - mean; pvar = fmaf(dlt, dlt, pvar); }
             stat[(2 + ch) * kRows + rr] = pvar;
-            asm volatile("bar.sync 1, 256;" ::: "memory");
+            asm volatile("bar.sync %0, 64;" ::"r"(1 + quad) : "memory");      // the two warps that share these 32 rows
             const float rstd = rsqrtf((stat[2 * kRows + rr] + stat[3 * kRows + rr]) * (1.f / kD) + eps);
 #pragma unroll
             for (int q16 = 0; q16 < 16; ++q16) {
