@@ -372,7 +372,8 @@ int Forward::run_t(const CallDesc &call, float *scores, cudaStream_t stream, std
             if constexpr (kTensor)
                 e = launch_attention_tc(tm_q, tm_k, tm_v, tm_pool, reinterpret_cast<const AttnItem *>(meta + o_items), (int)items.size(),
                                         reinterpret_cast<const AttnMerge *>(meta + o_merges), (int)merges.size(), d_seqs, meta + o_pt, L,
-                                        l, d, q, kl, vl, cfg.attn_kind, att, reinterpret_cast<float *>(ws + lay.partial), d_status, stream, &launches);
+                                        l, d, q, kl, vl, cfg.attn_kind, (!preinfer && l == L - 1) ? 1 : 0, att, reinterpret_cast<float *>(ws + lay.partial), d_status,
+                                        stream, &launches);
             else
                 e = launch_attention_simt<T>(q, kl, vl, paged, d_seqs, d_row_off, B, R, H, cfg.d_head, cfg.attn_kind, att, stream, &launches);
             prof_end(KC_ATTENTION, pe, stream);
