@@ -16,9 +16,15 @@ def _runtime():
     return binding, runtime
 
 
-def _setup(shape, seed, batch, hbm_pages=None, host_pages=0, page_ids=None):
+def _setup(shape, seed, batch, hbm_pages=None, host_pages=0, page_ids=None, q_gain=1.0):
     B, rt = _runtime()
     w = synth.make_weights(shape, seed)
+    if q_gain != 1.0:                                   # sharper (or flatter) attention logits; a power of two keeps bf16 values exact
+        d = shape.d_model
+        w.mat["w_qkv"][:, :d, :] *= np.float32(q_gain)
+        w.vec["b_qkv"][:, :d] *= np.float32(q_gain)
+        if "w_qkv" in w.bits:                           # the bf16 bit patterns are what the device gets
+            w.bits["w_qkv"] = synth.round_to_bf16_bits(w.mat["w_qkv"])
     model = rt.Model(shape, w)
     n_pages = [synth.pages_for(batch.prefix_off[i + 1] - batch.prefix_off[i]) for i in range(batch.n_users)]
     total = sum(n_pages)
@@ -458,4 +464,38 @@ def test_feed_forward_widths_d256(ff):
     assert max_abs_err(scores.cpu().numpy(), batch, want) <= TOL_BF16
     assert max_abs_err(full.cpu().numpy(), batch, want) <= TOL_BF16
     assert model.device_status() == 0
+    pool.close(); model.close()
+
+
+# ---------------------------------------------------------------- sharp attention logits: the softmax's slow path
+@pytest.mark.parametrize("q_gain", [8.0, 64.0])
+def test_sharp_logits_take_the_rescaling_path(q_gain):
+    """Queries scaled by 8 / 64: logits of tens to hundreds, nearly one-hot softmax rows.  The kernel's exponentials against a
+    stale running maximum overflow its row-sum check all the time here, so the block maximum, the rescaling of O and the
+    clamps of the FMA-pipe exponential all run.
+
+    What can be asked of the scores: Q and K are stored in bf16 (relative rounding 2^-9), so a logit of magnitude |s| carries an
+    absolute error of about |s| * 2^-8, and the softmax weights move by that fraction.  The logits grow with the gain, hence a
+    bound of gain * TOL_BF16 against the fp64 checker while the rows are not yet one-hot (gain 8).  At gain 64 a rounding of
+    that size decides which of two close keys takes the whole row, so single scores legitimately differ by O(1); there the
+    checks are the ones a broken slow path cannot pass: the typical (median) error stays small, and the cached rank and the
+    full recompute, which walk the keys in different block and split orders, agree with each other."""
+    shape = small_bf16_shape()
+    batch = _tiny_batch(shape, 111, [700, 130, 65], [40, 0, 9], [200, 33, 129])
+    w, model, pool, db = _setup(shape, 31, batch, q_gain=q_gain)
+    om = oracle_model(shape, w)
+    pool.preinfer(db)
+    scores = pool.rank(db).cpu().numpy()
+    full = model.rank_full(db).cpu().numpy()
+    torch.cuda.synchronize()
+    assert model.device_status() == 0
+    want = oracle_scores(om, batch)
+    if q_gain <= 8.0:
+        assert max_abs_err(scores, batch, want) <= q_gain * TOL_BF16
+        assert max_abs_err(full, batch, want) <= q_gain * TOL_BF16
+    else:
+        assert np.all(np.isfinite(scores)) and np.all(np.isfinite(full))
+        err = np.concatenate([np.abs(scores[batch.cand_off[i]:batch.cand_off[i + 1]] - wv) for i, wv in want.items()])
+        assert np.median(err) <= 0.1
+    assert np.max(np.abs(scores - full)) <= 4 * TOL_BF16
     pool.close(); model.close()
