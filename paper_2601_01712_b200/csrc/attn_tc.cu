@@ -38,6 +38,7 @@ constexpr int kStagesKV = 4;
 constexpr int kSmemBytes = kQBytes + 2 * kStagesKV * kKVBytes + 1024 + 512;
 constexpr uint32_t kTmemCols = 256;                 // S[2]: 0..127, P[2]: 128..191, O: 192..255
 constexpr uint32_t kColS = 0, kColP = 128, kColO = 192;
+constexpr int kPartStride = kDh + 4;                // floats per row of a split partial: m, l, two unused, then O (16-byte aligned rows)
 constexpr float kRowSumLimit = 256.f;               // a block's row sum above this: some p may exceed 2^8 -> redo against a raised maximum
 
 struct Bars {
@@ -467,10 +468,10 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                         dst[i] = w4;
                     }
                 } else {
-                    float *dst = partial + ((size_t)it.partial_slot * kQTile + r) * (kDh + 2);
-                    dst[0] = m; dst[1] = l;
+                    float4 *dst = reinterpret_cast<float4 *>(partial + ((size_t)it.partial_slot * kQTile + r) * kPartStride);
+                    dst[0] = make_float4(m, l, 0.f, 0.f);
 #pragma unroll
-                    for (int i = 0; i < kDh; ++i) dst[2 + i] = o[i];
+                    for (int i = 0; i < kDh / 4; ++i) dst[1 + i] = make_float4(o[4 * i], o[4 * i + 1], o[4 * i + 2], o[4 * i + 3]);
                 }
             }
         }
@@ -497,13 +498,13 @@ attention_merge_kernel(const AttnMerge *__restrict__ merges, const SeqDesc *__re
     const int r = blockIdx.y * 8 + warp;
     if (r < mg.n_q) {
         float M = -INFINITY;
-        for (int i = 0; i < mg.n_splits; ++i) M = fmaxf(M, partial[((size_t)(mg.slot0 + i) * kQTile + r) * (kDh + 2)]);
+        for (int i = 0; i < mg.n_splits; ++i) M = fmaxf(M, partial[((size_t)(mg.slot0 + i) * kQTile + r) * kPartStride]);
         float o0 = 0.f, o1 = 0.f, l = 0.f;
         for (int i = 0; i < mg.n_splits; ++i) {
-            const float *p = partial + ((size_t)(mg.slot0 + i) * kQTile + r) * (kDh + 2);
+            const float *p = partial + ((size_t)(mg.slot0 + i) * kQTile + r) * kPartStride;
             const float mi = p[0];
             const float wgt = (mi == -INFINITY) ? 0.f : ex2((mi - M) * c);
-            const float2 v = *reinterpret_cast<const float2 *>(p + 2 + 2 * lane);
+            const float2 v = *reinterpret_cast<const float2 *>(p + 4 + 2 * lane);
             l = fmaf(p[1], wgt, l);
             o0 = fmaf(v.x, wgt, o0);
             o1 = fmaf(v.y, wgt, o1);
@@ -522,12 +523,15 @@ cudaError_t launch_attention_tc(const CUtensorMap &tmQ, const CUtensorMap &tmK, 
                                 float *partial, int *err, cudaStream_t stream, int64_t *launches)
 {
     if (n_items == 0) return cudaSuccess;
-    static bool attr_set = false;
-    if (!attr_set) {
+    static PerDeviceValue attr_set;
+    int dev = 0;
+    cudaError_t e0 = cudaGetDevice(&dev);
+    if (e0 != cudaSuccess) return e0;
+    if (!attr_set.get(dev)) {
         cudaError_t e = cudaFuncSetAttribute(attention_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
         if (e == cudaSuccess) e = cudaFuncSetAttribute(attention_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
         if (e != cudaSuccess) return e;
-        attr_set = true;
+        attr_set.set(dev, 1);
     }
     *launches += 1;
     auto kernel = attn_kind == ATTN_POINTWISE ? attention_tc_kernel<true> : attention_tc_kernel<false>;

@@ -418,12 +418,15 @@ cudaError_t launch_ffn_fused(const CUtensorMap &tmW1, const CUtensorMap &tmW2, c
                              const float *bo, int64_t M, int d_ff, float eps, int *err, cudaStream_t stream, int64_t *launches)
 {
     if (M == 0) return cudaSuccess;
-    static bool attr_set = false;
-    if (!attr_set) {
+    static PerDeviceValue attr_set;
+    int dev = 0;
+    cudaError_t e0 = cudaGetDevice(&dev);
+    if (e0 != cudaSuccess) return e0;
+    if (!attr_set.get(dev)) {
         cudaError_t e = cudaFuncSetAttribute(ffn_fused_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
         if (e == cudaSuccess) e = cudaFuncSetAttribute(ffn_fused_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
         if (e != cudaSuccess) return e;
-        attr_set = true;
+        attr_set.set(dev, 1);
     }
     *launches += 1;
     const dim3 grid((unsigned)((M + kRows - 1) / kRows));

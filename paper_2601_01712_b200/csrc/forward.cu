@@ -128,7 +128,7 @@ WorkspaceLayout Forward::layout(int64_t rows, int64_t users, int64_t pages) cons
     l.v = take(r * d * es);
     l.att = take(r * d * es);
     l.hid = take(r * F * es);
-    l.partial_bytes = (size_t)kMaxSplitTiles * 128 * (size_t)(cfg.d_head + 2) * 4;
+    l.partial_bytes = (size_t)kMaxSplitTiles * 128 * (size_t)(cfg.d_head + 4) * 4;      // rows of m, l, two unused, O (see attention_merge_kernel)
     l.partial = take(l.partial_bytes);
     const size_t n_items = (size_t)cfg.n_heads * ((size_t)rows / 128 + (size_t)users + 1) + 2 * (size_t)kMaxSplitTiles;
     l.meta_bytes = 4 * (((size_t)users + 1) * 5 + (size_t)users * (sizeof(SeqDesc) / 4) + (size_t)pages + n_items * (sizeof(AttnItem) / 4) + 64);

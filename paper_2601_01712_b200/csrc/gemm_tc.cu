@@ -384,11 +384,14 @@ static cudaError_t launch_cfg(const CUtensorMap &tmA, const CUtensorMap &tmB, co
                               const Epilogue &epi, int *err, cudaStream_t stream)
 {
     using C = Cfg<BN, CTAS>;
-    static int n_workers_max = 0;                   // CTAs (or CTA pairs) that can be resident at once: one per SM (or SM pair)
+    static PerDeviceValue workers_of;               // CTAs (or CTA pairs) that can be resident at once: one per SM (or SM pair)
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    int n_workers_max = workers_of.get(dev);
     if (n_workers_max == 0) {
-        int dev = 0, n_sms = 0;
-        cudaError_t e = cudaGetDevice(&dev);
-        if (e == cudaSuccess) e = cudaDeviceGetAttribute(&n_sms, cudaDevAttrMultiProcessorCount, dev);
+        int n_sms = 0;
+        e = cudaDeviceGetAttribute(&n_sms, cudaDevAttrMultiProcessorCount, dev);
         if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_tc_kernel<BN, CTAS>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
         int n = n_sms / CTAS;
         if (e == cudaSuccess && CTAS == 2) {
@@ -405,6 +408,7 @@ static cudaError_t launch_cfg(const CUtensorMap &tmA, const CUtensorMap &tmB, co
         if (e != cudaSuccess) return e;
         if (n < 1) return cudaErrorLaunchOutOfResources;
         n_workers_max = n;
+        workers_of.set(dev, n);
     }
     const int64_t tiles = ((M + BM * CTAS - 1) / (BM * CTAS)) * (N / BN);
     const unsigned workers = (unsigned)(tiles < n_workers_max ? tiles : n_workers_max);

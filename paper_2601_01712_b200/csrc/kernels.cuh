@@ -4,6 +4,7 @@
 
 #include <cuda.h>
 
+#include <atomic>
 #include <utility>
 
 #include "internal.cuh"
@@ -30,6 +31,16 @@ cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, si
     }
     return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
 }
+
+// Once-per-device set-up of a kernel (opt-in shared memory size, occupancy query).  A function attribute belongs to the
+// device it was set on, so the launchers keep one slot per device: 0 = not set up yet, otherwise the value the set-up
+// produced.  Two threads that race through the set-up both store the same value.
+constexpr int kMaxDeviceSlots = 64;
+struct PerDeviceValue {
+    std::atomic<int> slot[kMaxDeviceSlots];
+    int get(int dev) const { return dev >= 0 && dev < kMaxDeviceSlots ? slot[dev].load(std::memory_order_acquire) : 0; }
+    void set(int dev, int v) { if (dev >= 0 && dev < kMaxDeviceSlots) slot[dev].store(v, std::memory_order_release); }
+};
 
 // ---- memory-bound steps (CUDA cores, vectorised loads, warp-shuffle reductions) ----------------
 
