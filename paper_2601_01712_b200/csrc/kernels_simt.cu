@@ -34,39 +34,6 @@ __device__ __forceinline__ void store4(__nv_bfloat16 *p, float4 v)
     *reinterpret_cast<uint2 *>(p) = u;
 }
 
-// LayerNorm of a row held in registers (chunks of 4 per lane), biased variance, fp32 statistics.
-template <typename T>
-__device__ __forceinline__ void ln_row_store(const float4 (&v)[kMaxChunks], int d, int lane, const float *g, const float *b,
-                                             float eps, T *out)
-{
-    float s = 0.f;
-#pragma unroll
-    for (int c = 0; c < kMaxChunks; ++c)
-        if ((c * 32 + lane) * 4 < d) s += v[c].x + v[c].y + v[c].z + v[c].w;
-    const float mean = warp_sum(s) / (float)d;
-    float q = 0.f;
-#pragma unroll
-    for (int c = 0; c < kMaxChunks; ++c)
-        if ((c * 32 + lane) * 4 < d) {
-            const float a0 = v[c].x - mean, a1 = v[c].y - mean, a2 = v[c].z - mean, a3 = v[c].w - mean;
-            q += a0 * a0 + a1 * a1 + a2 * a2 + a3 * a3;
-        }
-    const float rstd = rsqrtf(warp_sum(q) / (float)d + eps);
-#pragma unroll
-    for (int c = 0; c < kMaxChunks; ++c) {
-        const int i = (c * 32 + lane) * 4;
-        if (i < d) {
-            const float4 gg = load4(g + i), bb = load4(b + i);
-            float4 o;
-            o.x = (v[c].x - mean) * rstd * gg.x + bb.x;
-            o.y = (v[c].y - mean) * rstd * gg.y + bb.y;
-            o.z = (v[c].z - mean) * rstd * gg.z + bb.z;
-            o.w = (v[c].w - mean) * rstd * gg.w + bb.w;
-            store4(out + i, o);
-        }
-    }
-}
-
 __device__ __forceinline__ int row_token_id(const RowSource &src, int64_t row)
 {
     const int u = find_user(src.row_off, src.n_users, (int)row);
@@ -97,51 +64,12 @@ gather_rows_kernel(const T *__restrict__ emb, int64_t vocab, int d, const int32_
     for (int i = lane; i < n16; i += 32) o[i] = s[i];
 }
 
-template <typename T>
-__global__ void __launch_bounds__(kWarpsPerBlock * 32)
-gather_ln_kernel(const T *__restrict__ emb, int64_t vocab, int d, RowSource src, int64_t n_rows,
-                 const float *__restrict__ g, const float *__restrict__ b, float eps, float *__restrict__ x, T *__restrict__ a)
-{
-    grid_launch_dependents();
-    grid_dependency_wait();
-    const int64_t row = (int64_t)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
-    const int lane = threadIdx.x & 31;
-    if (row >= n_rows) return;
-    int64_t id = row_token_id(src, row);
-    id = id < 0 ? 0 : (id >= vocab ? vocab - 1 : id);
-    const T *e = emb + id * d;
-    float4 v[kMaxChunks];
-#pragma unroll
-    for (int c = 0; c < kMaxChunks; ++c) {
-        const int i = (c * 32 + lane) * 4;
-        if (i < d) {
-            v[c] = load4(e + i);
-            store4(x + row * d + i, v[c]);
-        }
-    }
-    ln_row_store<T>(v, d, lane, g, b, eps, a + row * d);
-}
-
-// a[r, :] = LN(x[r, :]).  A warp takes ROWS consecutive rows at once and issues all their loads before any
-// arithmetic, so that enough bytes are in flight per SM to reach HBM / L2 bandwidth; NC = chunks of 128 columns.
+// LayerNorm of ROWS rows a warp holds in registers (NC chunks of 128 columns, 4 values per lane and chunk; padding chunks
+// hold zeros), biased variance, fp32 statistics; rows from n_rows on are skipped.
 template <typename T, int NC, int ROWS>
-__global__ void __launch_bounds__(kWarpsPerBlock * 32)
-layernorm_kernel(const float *__restrict__ x, int d, int64_t n_rows, const float *__restrict__ g, const float *__restrict__ b,
-                 float eps, T *__restrict__ a)
+__device__ __forceinline__ void ln_rows_store(const float4 (&v)[ROWS][NC], int d, int lane, int64_t row0, int64_t n_rows,
+                                              const float *__restrict__ g, const float *__restrict__ b, float eps, T *__restrict__ a)
 {
-    grid_launch_dependents();
-    grid_dependency_wait();
-    const int64_t row0 = ((int64_t)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5)) * ROWS;
-    const int lane = threadIdx.x & 31;
-    if (row0 >= n_rows) return;
-    float4 v[ROWS][NC];
-#pragma unroll
-    for (int r = 0; r < ROWS; ++r)
-#pragma unroll
-        for (int c = 0; c < NC; ++c) {
-            const int i = (c * 32 + lane) * 4;
-            v[r][c] = (row0 + r < n_rows && i < d) ? load4(x + (row0 + r) * d + i) : make_float4(0.f, 0.f, 0.f, 0.f);
-        }
     float4 gg[NC], bb[NC];
 #pragma unroll
     for (int c = 0; c < NC; ++c) {
@@ -154,7 +82,7 @@ layernorm_kernel(const float *__restrict__ x, int d, int64_t n_rows, const float
         if (row0 + r >= n_rows) break;
         float s = 0.f;
 #pragma unroll
-        for (int c = 0; c < NC; ++c) s += (v[r][c].x + v[r][c].y) + (v[r][c].z + v[r][c].w);      // padding chunks hold zeros
+        for (int c = 0; c < NC; ++c) s += (v[r][c].x + v[r][c].y) + (v[r][c].z + v[r][c].w);
         const float mean = warp_sum(s) * inv_d;
         float q = 0.f;
 #pragma unroll
@@ -179,6 +107,72 @@ layernorm_kernel(const float *__restrict__ x, int d, int64_t n_rows, const float
     }
 }
 
+// x[r, :] = emb[id(r), :] widened to fp32, a[r, :] = LN(x[r, :]).  A warp takes ROWS consecutive rows: lane r walks the
+// look-up chain of row r (user of the row, segment, token id - dependent loads), so the ROWS chains run side by side, and
+// all table rows are requested before any arithmetic: the table rows are scattered over HBM, and one row per warp kept
+// too few bytes in flight.
+template <typename T, int NC, int ROWS>
+__global__ void __launch_bounds__(kWarpsPerBlock * 32)
+gather_ln_kernel(const T *__restrict__ emb, int64_t vocab, int d, RowSource src, int64_t n_rows,
+                 const float *__restrict__ g, const float *__restrict__ b, float eps, float *__restrict__ x, T *__restrict__ a)
+{
+    grid_launch_dependents();
+    grid_dependency_wait();
+    const int64_t row0 = ((int64_t)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5)) * ROWS;
+    const int lane = threadIdx.x & 31;
+    if (row0 >= n_rows) return;
+    long long my_id = 0;
+    if (lane < ROWS && row0 + lane < n_rows) {
+        my_id = row_token_id(src, row0 + lane);
+        my_id = my_id < 0 ? 0 : (my_id >= vocab ? vocab - 1 : my_id);
+    }
+    float4 v[ROWS][NC];
+#pragma unroll
+    for (int r = 0; r < ROWS; ++r) {
+        const T *e = emb + __shfl_sync(0xffffffffu, my_id, r) * d;
+#pragma unroll
+        for (int c = 0; c < NC; ++c) {
+            const int i = (c * 32 + lane) * 4;
+            v[r][c] = (row0 + r < n_rows && i < d) ? load4(e + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+    }
+#pragma unroll
+    for (int r = 0; r < ROWS; ++r)
+#pragma unroll
+        for (int c = 0; c < NC; ++c) {
+            const int i = (c * 32 + lane) * 4;
+            if (row0 + r < n_rows && i < d) store4(x + (row0 + r) * d + i, v[r][c]);
+        }
+    ln_rows_store<T, NC, ROWS>(v, d, lane, row0, n_rows, g, b, eps, a);
+}
+
+// a[r, :] = LN(x[r, :]).  A warp takes ROWS consecutive rows at once and issues all their loads before any
+// arithmetic, so that enough bytes are in flight per SM to reach HBM / L2 bandwidth; NC = chunks of 128 columns.
+template <typename T, int NC, int ROWS>
+__global__ void __launch_bounds__(kWarpsPerBlock * 32)
+layernorm_kernel(const float *__restrict__ x, int d, int64_t n_rows, const float *__restrict__ g, const float *__restrict__ b,
+                 float eps, T *__restrict__ a)
+{
+    grid_launch_dependents();
+    grid_dependency_wait();
+    const int64_t row0 = ((int64_t)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5)) * ROWS;
+    const int lane = threadIdx.x & 31;
+    if (row0 >= n_rows) return;
+    float4 v[ROWS][NC];
+#pragma unroll
+    for (int r = 0; r < ROWS; ++r)
+#pragma unroll
+        for (int c = 0; c < NC; ++c) {
+            const int i = (c * 32 + lane) * 4;
+            v[r][c] = (row0 + r < n_rows && i < d) ? load4(x + (row0 + r) * d + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+    ln_rows_store<T, NC, ROWS>(v, d, lane, row0, n_rows, g, b, eps, a);
+}
+
+// score[i] = w . LN(x[row(i), :]; g, b) + bias for the candidate rows.  As in the kernels above a warp takes ROWS
+// consecutive candidates, lane r resolves candidate r's row (user look-up: dependent loads), and all rows are requested
+// before any arithmetic.
+template <int NC, int ROWS>
 __global__ void __launch_bounds__(kWarpsPerBlock * 32)
 score_kernel(const float *__restrict__ x, int d, const SeqDesc *__restrict__ seqs, int n_users, int64_t n_total,
              const int32_t *__restrict__ score_off, const float *__restrict__ g, const float *__restrict__ b, float eps,
@@ -186,42 +180,56 @@ score_kernel(const float *__restrict__ x, int d, const SeqDesc *__restrict__ seq
 {
     grid_launch_dependents();
     grid_dependency_wait();
-    const int64_t idx = (int64_t)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
+    const int64_t idx0 = ((int64_t)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5)) * ROWS;
     const int lane = threadIdx.x & 31;
-    if (idx >= n_total) return;
-    const int u = find_user(score_off, n_users, (int)idx);
-    const int64_t row = (int64_t)seqs[u].score_row0 + ((int)idx - score_off[u]);
-    float4 v[kMaxChunks];
-    float s = 0.f;
+    if (idx0 >= n_total) return;
+    long long my_row = 0;
+    if (lane < ROWS && idx0 + lane < n_total) {
+        const int idx = (int)(idx0 + lane);
+        const int u = find_user(score_off, n_users, idx);
+        my_row = (long long)seqs[u].score_row0 + (idx - score_off[u]);
+    }
+    float4 v[ROWS][NC];
 #pragma unroll
-    for (int c = 0; c < kMaxChunks; ++c) {
-        const int i = (c * 32 + lane) * 4;
-        if (i < d) {
-            v[c] = load4(x + row * d + i);
-            s += v[c].x + v[c].y + v[c].z + v[c].w;
+    for (int r = 0; r < ROWS; ++r) {
+        const float *xr = x + __shfl_sync(0xffffffffu, my_row, r) * d;
+#pragma unroll
+        for (int c = 0; c < NC; ++c) {
+            const int i = (c * 32 + lane) * 4;
+            v[r][c] = (idx0 + r < n_total && i < d) ? load4(xr + i) : make_float4(0.f, 0.f, 0.f, 0.f);
         }
     }
-    const float mean = warp_sum(s) / (float)d;
-    float q = 0.f;
+    float4 gg[NC], bb[NC], ww[NC];
 #pragma unroll
-    for (int c = 0; c < kMaxChunks; ++c)
-        if ((c * 32 + lane) * 4 < d) {
-            const float a0 = v[c].x - mean, a1 = v[c].y - mean, a2 = v[c].z - mean, a3 = v[c].w - mean;
-            q += a0 * a0 + a1 * a1 + a2 * a2 + a3 * a3;
-        }
-    const float rstd = rsqrtf(warp_sum(q) / (float)d + eps);
-    float acc = 0.f;
-#pragma unroll
-    for (int c = 0; c < kMaxChunks; ++c) {
+    for (int c = 0; c < NC; ++c) {
         const int i = (c * 32 + lane) * 4;
-        if (i < d) {
-            const float4 gg = load4(g + i), bb = load4(b + i), ww = load4(w + i);
-            acc += ((v[c].x - mean) * rstd * gg.x + bb.x) * ww.x + ((v[c].y - mean) * rstd * gg.y + bb.y) * ww.y +
-                   ((v[c].z - mean) * rstd * gg.z + bb.z) * ww.z + ((v[c].w - mean) * rstd * gg.w + bb.w) * ww.w;
-        }
+        if (i < d) { gg[c] = load4(g + i); bb[c] = load4(b + i); ww[c] = load4(w + i); }
     }
-    acc = warp_sum(acc);
-    if (lane == 0) scores[idx] = acc + (bias ? bias[0] : 0.f);
+    const float inv_d = 1.f / (float)d, bias0 = bias ? bias[0] : 0.f;
+#pragma unroll
+    for (int r = 0; r < ROWS; ++r) {
+        if (idx0 + r >= n_total) break;
+        float s = 0.f;
+#pragma unroll
+        for (int c = 0; c < NC; ++c) s += (v[r][c].x + v[r][c].y) + (v[r][c].z + v[r][c].w);
+        const float mean = warp_sum(s) * inv_d;
+        float q = 0.f;
+#pragma unroll
+        for (int c = 0; c < NC; ++c)
+            if ((c * 32 + lane) * 4 < d) {
+                const float a0 = v[r][c].x - mean, a1 = v[r][c].y - mean, a2 = v[r][c].z - mean, a3 = v[r][c].w - mean;
+                q += a0 * a0 + a1 * a1 + a2 * a2 + a3 * a3;
+            }
+        const float rstd = rsqrtf(warp_sum(q) * inv_d + eps);
+        float acc = 0.f;
+#pragma unroll
+        for (int c = 0; c < NC; ++c)
+            if ((c * 32 + lane) * 4 < d)
+                acc += ((v[r][c].x - mean) * rstd * gg[c].x + bb[c].x) * ww[c].x + ((v[r][c].y - mean) * rstd * gg[c].y + bb[c].y) * ww[c].y +
+                       ((v[r][c].z - mean) * rstd * gg[c].z + bb[c].z) * ww[c].z + ((v[r][c].w - mean) * rstd * gg[c].w + bb[c].w) * ww[c].w;
+        acc = warp_sum(acc);
+        if (lane == 0) scores[idx0 + r] = acc + bias0;
+    }
 }
 
 // ---- epilogue shared by the CUDA-core GEMM (one element at a time) ----------------------------------
@@ -389,9 +397,18 @@ cudaError_t launch_gather_ln(const T *emb, int64_t vocab, int d, RowSource src, 
                              const float *b, float eps, float *x, T *a, cudaStream_t stream, int64_t *launches)
 {
     if (n_rows == 0) return cudaSuccess;
+    const int nc = (d + 127) / 128;
+    cudaError_t e;
+#define RELAYGR_GLN(NC, ROWS)                                                                                             \
+    e = launch_dependent(gather_ln_kernel<T, NC, ROWS>, dim3(blocks_for((n_rows + ROWS - 1) / ROWS)), dim3(kWarpsPerBlock * 32), 0, stream, 1, \
+                         emb, vocab, d, src, n_rows, g, b, eps, x, a)
+    if (nc <= 1) RELAYGR_GLN(1, 4);
+    else if (nc <= 2) RELAYGR_GLN(2, 4);
+    else if (nc <= 4) RELAYGR_GLN(4, 4);
+    else RELAYGR_GLN(8, 1);
+#undef RELAYGR_GLN
     *launches += 1;
-    return launch_dependent(gather_ln_kernel<T>, dim3(blocks_for(n_rows)), dim3(kWarpsPerBlock * 32), 0, stream, 1, emb, vocab, d, src, n_rows, g,
-                            b, eps, x, a);
+    return e;
 }
 
 template <typename T>
@@ -418,9 +435,18 @@ cudaError_t launch_score(const float *x, int d, const SeqDesc *seqs, int n_users
                          cudaStream_t stream, int64_t *launches)
 {
     if (n_total == 0) return cudaSuccess;
+    const int nc = (d + 127) / 128;
+    cudaError_t e;
+#define RELAYGR_SCORE(NC, ROWS)                                                                                           \
+    e = launch_dependent(score_kernel<NC, ROWS>, dim3(blocks_for((n_total + ROWS - 1) / ROWS)), dim3(kWarpsPerBlock * 32), 0, stream, 1, x, d, \
+                         seqs, n_users, n_total, score_off, g, b, eps, w, bias, scores)
+    if (nc <= 1) RELAYGR_SCORE(1, 4);
+    else if (nc <= 2) RELAYGR_SCORE(2, 4);
+    else if (nc <= 4) RELAYGR_SCORE(4, 2);
+    else RELAYGR_SCORE(8, 1);
+#undef RELAYGR_SCORE
     *launches += 1;
-    return launch_dependent(score_kernel, dim3(blocks_for(n_total)), dim3(kWarpsPerBlock * 32), 0, stream, 1, x, d, seqs, n_users, n_total,
-                            score_off, g, b, eps, w, bias, scores);
+    return e;
 }
 
 template <typename T>
