@@ -499,3 +499,55 @@ def test_sharp_logits_take_the_rescaling_path(q_gain):
         assert np.median(err) <= 0.1
     assert np.max(np.abs(scores - full)) <= 4 * TOL_BF16
     pool.close(); model.close()
+
+
+# ---------------------------------------------------------------- randomized shapes around the tile, page and warp boundaries
+_EDGE_LENGTHS = [1, 2, 31, 32, 33, 63, 64, 65, 127, 128, 129, 191, 192, 193, 255, 256, 257, 511, 512, 513, 1023, 1024, 1025]
+
+
+def _random_case(rng):
+    def pick(lo, hi, allow_zero=False):
+        r = rng.random()
+        if allow_zero and r < 0.15:
+            return 0
+        if r < 0.5:
+            return int(rng.choice([e for e in _EDGE_LENGTHS if lo <= e <= hi]))
+        return int(rng.integers(lo, hi + 1))
+    d = int(rng.choice([128, 256, 256, 256, 384, 512]))
+    layers = int(rng.integers(1, 4))
+    ff = int(rng.choice([128, 256, 512, 1024])) if d == 256 else (4 * d if rng.random() < 0.5 else int(rng.choice([128, 384, 640])))
+    kind = int(rng.random() < 0.25)
+    n = int(rng.integers(1, 6))
+    return d, layers, ff, kind, [pick(1, 1300) for _ in range(n)], [pick(1, 200, True) for _ in range(n)], [pick(1, 300, True) for _ in range(n)]
+
+
+@pytest.mark.parametrize("block", range(4))
+def test_randomized_shapes_match_checker(block):
+    """Seeded random models (width, depth, feed-forward width, attention variant) and jagged batches whose lengths cluster
+    around the boundaries of the 64-token pages, the 128-row query tiles and the 32-row warps, half of them on shuffled
+    pages.  The error against the checker behaves like noise of rms 0.004-0.005 on scores of unit scale (bf16 rounding of
+    the activations), whose tail over a few hundred candidates reaches 4-4.5 rms: the bound on the maximum is 1.5 x the bf16
+    tolerance of the named workloads, with the rms bounded as well, so that a systematic error does not hide under it."""
+    rng = np.random.default_rng(9100 + block)
+    for it in range(6):
+        d, layers, ff, kind, p, s, c = _random_case(rng)
+        shape = small_bf16_shape(vocab=3000, layers=layers, d=d, heads=d // 64, ff=ff, attn_kind=kind)
+        batch = _tiny_batch(shape, 1000 * block + it, p, s, c)
+        counts = [synth.pages_for(x) for x in p]
+        ids = synth.shuffled_pages(np.random.default_rng(it), sum(counts) + 7, counts) if rng.random() < 0.5 else None
+        w, model, pool, db = _setup(shape, 500 + 10 * block + it, batch, hbm_pages=sum(counts) + 7, page_ids=ids)
+        om = oracle_model(shape, w)
+        pool.preinfer(db)
+        scores = pool.rank(db).cpu().numpy()
+        full = model.rank_full(db).cpu().numpy()
+        torch.cuda.synchronize()
+        assert model.device_status() == 0
+        want = oracle_scores(om, batch)
+        tol = TOL_BF16_POINTWISE if kind else TOL_BF16
+        case = (d, layers, ff, kind, p, s, c)
+        for got in (scores, full):
+            assert max_abs_err(got, batch, want) <= 1.5 * tol, case
+            err = np.concatenate([got[batch.cand_off[i]:batch.cand_off[i + 1]] - wv for i, wv in want.items()])
+            if len(err):
+                assert np.sqrt(np.mean(err ** 2)) <= 0.4 * tol, case
+        pool.close(); model.close()
