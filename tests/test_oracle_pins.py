@@ -65,31 +65,68 @@ def test_brute_force_three_heads_one_layer():
 
 
 # ---------------------------------------------------------------- (2) textbook special case
-def test_causal_special_case_against_library_attention():
-    """S = 0, C = 1: an ordinary causal pre-LN transformer read at its last token."""
-    shape = tiny_shape(L=2, d=16, H=2, F=32)
-    m, params = make_model(shape, 5)
-    rng = np.random.default_rng(11)
-    p, c = ids(rng, 13), ids(rng, 1)
-    got = m.full(p, np.zeros(0, np.int32), c)[0]
-
+def library_last_token_score(shape, params, ids_all, attn_mask=None):
+    """A pre-LN transformer over one token sequence, written with torch's library routines and read at its
+    last token.  attn_mask = None: ordinary causal attention (is_causal=True); else a boolean [T, T] mask."""
     t = lambda a: torch.tensor(np.asarray(a), dtype=torch.float64)
     d, H, dh = shape.d_model, shape.n_heads, shape.d_head
-    x = t(params["emb"])[torch.tensor(np.concatenate([p, c]).astype(np.int64))]
+    x = t(params["emb"])[torch.tensor(np.asarray(ids_all).astype(np.int64))]
     T = x.shape[0]
     for l in range(shape.n_layers):
         a = torch.nn.functional.layer_norm(x, (d,), t(params["ln1_g"][l]), t(params["ln1_b"][l]), shape.ln_eps)
         qkv = torch.nn.functional.linear(a, t(params["w_qkv"][l]), t(params["b_qkv"][l]))
         q, k, v = [z.reshape(T, H, dh).transpose(0, 1) for z in qkv.split(d, dim=1)]
-        o = torch.nn.functional.scaled_dot_product_attention(q, k, v, is_causal=True)
+        if attn_mask is None:
+            o = torch.nn.functional.scaled_dot_product_attention(q, k, v, is_causal=True)
+        else:
+            o = torch.nn.functional.scaled_dot_product_attention(q, k, v, attn_mask=torch.tensor(attn_mask))
         o = o.transpose(0, 1).reshape(T, d)
         h = x + torch.nn.functional.linear(o, t(params["w_o"][l]), t(params["b_o"][l]))
         a2 = torch.nn.functional.layer_norm(h, (d,), t(params["ln2_g"][l]), t(params["ln2_b"][l]), shape.ln_eps)
         z = torch.nn.functional.silu(torch.nn.functional.linear(a2, t(params["w1"][l]), t(params["b1"][l])))
         x = h + torch.nn.functional.linear(z, t(params["w2"][l]), t(params["b2"][l]))
     a = torch.nn.functional.layer_norm(x[-1], (d,), t(params["lnf_g"]), t(params["lnf_b"]), shape.ln_eps)
-    want = float(a @ t(params["w_score"]) + float(params["b_score"][0]))
+    return float(a @ t(params["w_score"]) + float(params["b_score"][0]))
+
+
+@pytest.mark.parametrize("P,S", [(13, 0), (9, 5), (1, 7), (6, 1)])
+def test_causal_special_case_against_library_attention(P, S):
+    """C = 1: [prefix; short-term; one candidate] is an ordinary causal sequence (every token sees exactly the
+    tokens up to itself), so the candidate's score is a plain causal pre-LN transformer read at its last
+    token.  With S > 0 this pins the short-term rows' causal edge, through every layer, against the library's
+    own causal mask - a writing of the mask that shares nothing with the checker's or the brute force's."""
+    shape = tiny_shape(L=2, d=16, H=2, F=32)
+    m, params = make_model(shape, 5)
+    rng = np.random.default_rng(11 + P + 31 * S)
+    p, s, c = ids(rng, P), ids(rng, S), ids(rng, 1)
+    got = m.full(p, s, c)[0]
+    want = library_last_token_score(shape, params, np.concatenate([p, s, c]))
     assert abs(got - want) <= 1e-10
+    K, V = m.preinfer(p)
+    assert abs(m.rank_cached(K, V, s, c)[0] - want) <= 1e-10
+
+
+@pytest.mark.parametrize("mistake", ["short_sees_later_short", "short_misses_itself", "short_misses_prefix"])
+def test_library_pin_catches_a_wrong_short_term_edge(mistake):
+    """The same library computation with the short-term rows' mask edge moved the way a plausible bug would
+    move it: the candidate's score then differs from the checker's by far more than the pin's 1e-10, so a
+    checker with that bug fails test_causal_special_case_against_library_attention."""
+    shape = tiny_shape(L=2, d=16, H=2, F=32)
+    m, params = make_model(shape, 5)
+    rng = np.random.default_rng(12)
+    P, S = 9, 5
+    p, s, c = ids(rng, P), ids(rng, S), ids(rng, 1)
+    T = P + S + 1
+    mask = np.tril(np.ones((T, T), dtype=bool))
+    assert abs(m.full(p, s, c)[0] - library_last_token_score(shape, params, np.concatenate([p, s, c]), mask)) <= 1e-10
+    if mistake == "short_sees_later_short":
+        mask[P:P + S, P:P + S] = True
+    elif mistake == "short_misses_itself":
+        mask[P:P + S, P:P + S] &= ~np.eye(S, dtype=bool)
+    else:
+        mask[P:P + S, :P] = False
+    wrong = library_last_token_score(shape, params, np.concatenate([p, s, c]), mask)
+    assert abs(m.full(p, s, c)[0] - wrong) > 1e-4
 
 
 # ---------------------------------------------------------------- (3) defining relation
