@@ -196,8 +196,21 @@ int32_t relaygr_kv_alloc(relaygr_kv_pool *pool, uint64_t user, int32_t prefix_le
  * and copied into the pages returned by relaygr_kv_pages, by work already enqueued
  * on `stream`): the entry becomes HBM-resident, ordered behind that stream's work.
  * E_MISS if unknown, E_INVALID if not ALLOCATED.
+ * The pages may have belonged to another user whose spill copy or last rank is still
+ * running: call relaygr_kv_wait_pages(pool, user, stream) BEFORE enqueueing the writes.
+ * Slots of the last page past prefix_len are never unmasked, but the attention kernels
+ * multiply them by a weight of zero: they must hold finite values (zeros will do).
  */
 int32_t relaygr_kv_commit(relaygr_kv_pool *pool, uint64_t user, void *stream);
+
+/*
+ * Make `stream` wait until every earlier owner of the user's HBM pages has finished with
+ * them (Section 3.3: pages change hands as the window slides; a freed page is handed out
+ * at once, behind the events of its earlier owners' copies and kernels).  relaygr_preinfer
+ * and relaygr_kv_reload_from_host do this themselves; a caller that writes pages directly
+ * (relaygr_kv_commit) must.  Enqueues stream waits only.  E_MISS if unknown.
+ */
+int32_t relaygr_kv_wait_pages(relaygr_kv_pool *pool, uint64_t user, void *stream);
 
 /* Drop the user's entry in every tier.  E_MISS if unknown, E_BUSY while LOADING. */
 int32_t relaygr_kv_free(relaygr_kv_pool *pool, uint64_t user);
@@ -230,11 +243,31 @@ int32_t relaygr_kv_lookup(relaygr_kv_pool *pool, uint64_t user, int32_t *tier, i
 int32_t relaygr_kv_pages(relaygr_kv_pool *pool, uint64_t user, int32_t *page_ids_out, int32_t cap, int32_t *n_out);
 int32_t relaygr_kv_stats(relaygr_kv_pool *pool, relaygr_pool_stats *out);
 
+/*
+ * Test control of a host-only pool (relaygr_create_host_only), so that the states of Section 3.4
+ * that need time on a GPU - a reload in flight, pages waiting for a spill copy, the bound on
+ * concurrent reloads, a failed transfer - can be held and checked without one.
+ *   MANUAL_EVENTS   arg != 0: events recorded from now on stay pending until completed below
+ *   COMPLETE_EVENTS complete the arg oldest pending events (arg < 0: all); *out = how many
+ *   FAIL_COPIES     the next arg tier copies fail (as a failed cudaMemcpyAsync would)
+ *   STREAM_WAITS    *out = number of "stream waits for event" requests the pool has made
+ *   PENDING_EVENTS  *out = number of pending events
+ * out may be NULL.  E_UNSUPPORTED on a pool that lives on a GPU, E_INVALID for an unknown request.
+ */
+enum {
+    RELAYGR_HOSTCTL_MANUAL_EVENTS = 0,
+    RELAYGR_HOSTCTL_COMPLETE_EVENTS = 1,
+    RELAYGR_HOSTCTL_FAIL_COPIES = 2,
+    RELAYGR_HOSTCTL_STREAM_WAITS = 3,
+    RELAYGR_HOSTCTL_PENDING_EVENTS = 4
+};
+int32_t relaygr_kv_host_backend_control(relaygr_kv_pool *pool, int32_t what, int64_t arg, int64_t *out);
+
 /* ---- the hot path -------------------------------------------------------------------------- */
 
 /*
- * Step P1/R2 alone: out[i, :] = emb[ids[i], :] for n ids, a bit-exact row copy
- * in cfg.dtype.  ids dev int32 [n], out dev [n, d].
+ * The embedding gather alone (the first step of both passes): out[i, :] = emb[ids[i], :]
+ * for n ids, a bit-exact row copy in cfg.dtype.  ids dev int32 [n], out dev [n, d].
  */
 int32_t relaygr_gather(relaygr_ctx *ctx, const int32_t *ids, int64_t n, void *out, void *stream);
 

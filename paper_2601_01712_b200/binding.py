@@ -75,6 +75,8 @@ SIGNATURES = {
     "relaygr_kv_set_max_inflight_reloads": (_I32, [_P, _I32]),
     "relaygr_kv_alloc": (_I32, [_P, _U64, _I32, _P]),
     "relaygr_kv_commit": (_I32, [_P, _U64, _P]),
+    "relaygr_kv_wait_pages": (_I32, [_P, _U64, _P]),
+    "relaygr_kv_host_backend_control": (_I32, [_P, _I32, _I64, C.POINTER(_I64)]),
     "relaygr_kv_free": (_I32, [_P, _U64]),
     "relaygr_kv_evict": (_I32, [_P, _U64, _I32, _P]),
     "relaygr_kv_reload_from_host": (_I32, [_P, _U64, _P, C.POINTER(_P)]),
@@ -199,6 +201,20 @@ def relaygr_kv_alloc(pool, user, prefix_len, page_ids=None, ok=(OK,)) -> int:
 
 def relaygr_kv_commit(pool, user, stream=None, ok=(OK,)) -> int:
     return _check(lib().relaygr_kv_commit(pool, user, stream), ok)
+
+
+def relaygr_kv_wait_pages(pool, user, stream=None, ok=(OK,)) -> int:
+    return _check(lib().relaygr_kv_wait_pages(pool, user, stream), ok)
+
+
+HOSTCTL_MANUAL_EVENTS, HOSTCTL_COMPLETE_EVENTS, HOSTCTL_FAIL_COPIES, HOSTCTL_STREAM_WAITS, HOSTCTL_PENDING_EVENTS = range(5)
+
+
+def relaygr_kv_host_backend_control(pool, what, arg=0, ok=(OK,)):
+    """Returns (status, value) of a test-control request to a host-only pool."""
+    out = _I64(0)
+    code = _check(lib().relaygr_kv_host_backend_control(pool, what, arg, C.byref(out)), ok)
+    return code, out.value
 
 
 def relaygr_kv_free(pool, user, ok=(OK,)) -> int:

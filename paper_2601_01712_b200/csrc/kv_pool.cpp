@@ -6,17 +6,54 @@
 namespace relaygr {
 
 namespace {
-// Host-only backend: tiers are plain host memory, copies are synchronous, events are always complete.
+// Host-only backend: tiers are plain host memory and copies are synchronous.  Events complete at once, unless a test
+// has switched to manual mode: then a recorded event stays pending until the test completes it, so that the states
+// that need time on a GPU (LOADING, pages waiting for a spill) can be held and looked at.  Copies can be told to fail.
 struct HostBackend : Backend {
+    struct Ev { bool pending = false; };
     bool is_cuda() const override { return false; }
-    int copy_h2d(void *dst, const void *src, size_t bytes, void *) override { std::memcpy(dst, src, bytes); return 0; }
-    int copy_d2h(void *dst, const void *src, size_t bytes, void *) override { std::memcpy(dst, src, bytes); return 0; }
-    void *event_create() override { return (void *)&token_; }
-    void event_destroy(void *) override {}
-    int event_record(void *, void *) override { return 0; }
-    bool event_done(void *) override { return true; }
-    int stream_wait(void *, void *) override { return 0; }
-    int token_ = 0;
+    int copy(void *dst, const void *src, size_t bytes)
+    {
+        if (fail_copies_ > 0) { --fail_copies_; return -1; }
+        std::memcpy(dst, src, bytes);
+        return 0;
+    }
+    int copy_h2d(void *dst, const void *src, size_t bytes, void *) override { return copy(dst, src, bytes); }
+    int copy_d2h(void *dst, const void *src, size_t bytes, void *) override { return copy(dst, src, bytes); }
+    void *event_create() override { return new Ev(); }
+    void event_destroy(void *ev) override
+    {
+        pending_.erase(std::remove(pending_.begin(), pending_.end(), (Ev *)ev), pending_.end());
+        delete (Ev *)ev;
+    }
+    int event_record(void *ev, void *) override
+    {
+        Ev *e = (Ev *)ev;
+        pending_.erase(std::remove(pending_.begin(), pending_.end(), e), pending_.end());
+        e->pending = manual_;
+        if (manual_) pending_.push_back(e);
+        return 0;
+    }
+    bool event_done(void *ev) override { return !((Ev *)ev)->pending; }
+    int stream_wait(void *, void *) override { ++stream_waits_; return 0; }
+    int64_t control(int32_t what, int64_t arg) override
+    {
+        switch (what) {
+            case RELAYGR_HOSTCTL_MANUAL_EVENTS: manual_ = arg != 0; return 0;
+            case RELAYGR_HOSTCTL_COMPLETE_EVENTS: {
+                int64_t n = 0;
+                while (!pending_.empty() && (arg < 0 || n < arg)) { pending_.front()->pending = false; pending_.erase(pending_.begin()); ++n; }
+                return n;
+            }
+            case RELAYGR_HOSTCTL_FAIL_COPIES: fail_copies_ = arg < 0 ? 0 : arg; return 0;
+            case RELAYGR_HOSTCTL_STREAM_WAITS: return stream_waits_;
+            case RELAYGR_HOSTCTL_PENDING_EVENTS: return (int64_t)pending_.size();
+        }
+        return RELAYGR_E_INVALID;
+    }
+    bool manual_ = false;
+    int64_t fail_copies_ = 0, stream_waits_ = 0;
+    std::vector<Ev *> pending_;      // in record order
 };
 }  // namespace
 
@@ -30,7 +67,8 @@ KvPool::KvPool(Backend *be, const relaygr_model_cfg &cfg, void *hbm, size_t hbm_
     n_pages_ = (int64_t)(hbm_bytes / page_bytes_);
     n_host_pages_ = host ? (int64_t)(host_bytes / page_bytes_) : 0;
     page_used_.assign((size_t)n_pages_, 0);
-    page_release_ticket_.assign((size_t)n_pages_, -1);
+    page_release_.assign((size_t)n_pages_, std::vector<int64_t>());
+    host_release_.assign((size_t)n_host_pages_, -1);
     free_pages_.reserve((size_t)n_pages_);
     for (int64_t p = n_pages_ - 1; p >= 0; --p) free_pages_.push_back((int32_t)p);   // pop_back hands out 0, 1, 2, ...
     free_host_.reserve((size_t)n_host_pages_);
@@ -104,13 +142,55 @@ int KvPool::wait_pages_released(void *stream, const std::vector<int32_t> &pages)
 {
     std::vector<int64_t> seen;
     for (int32_t p : pages) {
-        const int64_t t = page_release_ticket_[(size_t)p];
+        std::vector<int64_t> &list = page_release_[(size_t)p];
+        size_t keep = 0;
+        for (int64_t t : list) {
+            if (ticket_done(t)) continue;
+            list[keep++] = t;
+            if (std::find(seen.begin(), seen.end(), t) != seen.end()) continue;
+            seen.push_back(t);
+            if (wait_ticket(stream, t) != 0) return RELAYGR_E_CUDA;
+        }
+        list.resize(keep);
+    }
+    return 0;
+}
+
+int KvPool::wait_host_pages_released(void *stream, const std::vector<int32_t> &pages)
+{
+    std::vector<int64_t> seen;
+    for (int32_t p : pages) {
+        const int64_t t = host_release_[(size_t)p];
         if (t < 0) continue;
-        if (ticket_done(t)) { page_release_ticket_[(size_t)p] = -1; continue; }
+        if (ticket_done(t)) { host_release_[(size_t)p] = -1; continue; }
         if (std::find(seen.begin(), seen.end(), t) != seen.end()) continue;
         seen.push_back(t);
         if (wait_ticket(stream, t) != 0) return RELAYGR_E_CUDA;
     }
+    return 0;
+}
+
+void KvPool::add_use(UserEntry &e, int64_t ticket)
+{
+    size_t keep = 0;
+    for (int64_t t : e.use_tickets) if (!ticket_done(t)) e.use_tickets[keep++] = t;
+    e.use_tickets.resize(keep);
+    if (ticket >= 0) e.use_tickets.push_back(ticket);
+}
+
+std::vector<int64_t> KvPool::pending_of(UserEntry &e)
+{
+    std::vector<int64_t> out;
+    if (e.ready_ticket >= 0 && !ticket_done(e.ready_ticket)) out.push_back(e.ready_ticket);
+    for (int64_t t : e.use_tickets) if (!ticket_done(t) && std::find(out.begin(), out.end(), t) == out.end()) out.push_back(t);
+    return out;
+}
+
+int KvPool::wait_pages_of(uint64_t user, void *stream, std::string &err)
+{
+    UserEntry *e = find(user);
+    if (!e) { err = "kv_wait_pages: unknown user"; return RELAYGR_E_MISS; }
+    if (wait_pages_released(stream, e->pages) != 0) { err = "kv_wait_pages: could not make the stream wait"; return RELAYGR_E_CUDA; }
     return 0;
 }
 
@@ -152,11 +232,17 @@ int KvPool::take_pages(int32_t n, const int32_t *ids, std::vector<int32_t> &out,
     return 0;
 }
 
-void KvPool::release_pages(std::vector<int32_t> &pages, int64_t ticket)
+void KvPool::release_pages(std::vector<int32_t> &pages, const std::vector<int64_t> &behind)
 {
     for (auto it = pages.rbegin(); it != pages.rend(); ++it) {
         page_used_[(size_t)*it] = 0;
-        page_release_ticket_[(size_t)*it] = ticket;
+        // what an earlier owner left pending stays: the entry that releases now may never have run anything on the page
+        std::vector<int64_t> &list = page_release_[(size_t)*it];
+        size_t keep = 0;
+        for (int64_t t : list) if (!ticket_done(t)) list[keep++] = t;
+        list.resize(keep);
+        for (int64_t t : behind)
+            if (t >= 0 && !ticket_done(t) && std::find(list.begin(), list.end(), t) == list.end()) list.push_back(t);
         free_pages_.push_back(*it);
     }
     pages.clear();
@@ -168,6 +254,15 @@ void KvPool::release_pages(std::vector<int32_t> &pages, int64_t ticket)
         for (int32_t p : free_pages_) if (!page_used_[(size_t)p] && !seen[(size_t)p]) { seen[(size_t)p] = 1; keep.push_back(p); }
         free_pages_.swap(keep);
     }
+}
+
+void KvPool::release_host_pages(std::vector<int32_t> &pages, int64_t behind)
+{
+    for (int32_t p : pages) {
+        host_release_[(size_t)p] = (behind >= 0 && !ticket_done(behind)) ? behind : -1;
+        free_host_.push_back(p);
+    }
+    pages.clear();
 }
 
 int KvPool::copy_pages(bool to_host, const std::vector<int32_t> &dev, const std::vector<int32_t> &host, void *stream)
@@ -221,8 +316,8 @@ int KvPool::free_user(uint64_t user, std::string &err)
     UserEntry *e = find(user);
     if (!e) { err = "kv_free: unknown user"; return RELAYGR_E_MISS; }
     if (tier_of(*e) == RELAYGR_TIER_LOADING) { err = "kv_free: reload in flight"; return RELAYGR_E_BUSY; }
-    release_pages(e->pages, e->last_use_ticket);
-    for (int32_t p : e->host_pages) free_host_.push_back(p);
+    release_pages(e->pages, pending_of(*e));
+    release_host_pages(e->host_pages, e->host_ticket);      // a spill copy may still be writing them
     users_.erase(user);
     return 0;
 }
@@ -235,11 +330,11 @@ int KvPool::evict(uint64_t user, bool spill, void *side, std::string &err)
     if (tier == RELAYGR_TIER_LOADING) { err = "kv_evict: reload in flight"; return RELAYGR_E_BUSY; }
     if (tier == RELAYGR_TIER_HOST) { err = "kv_evict: user holds no HBM pages"; return RELAYGR_E_MISS; }
     if (tier == RELAYGR_TIER_ALLOCATED) {            // nothing was computed yet: just give the pages back
-        release_pages(e->pages, e->last_use_ticket);
+        release_pages(e->pages, pending_of(*e));
         users_.erase(user);
         return 0;
     }
-    int64_t release_after = e->last_use_ticket;
+    std::vector<int64_t> release_after = pending_of(*e);
     if (spill && e->host_pages.empty()) {
         if (!host_ || (int64_t)free_host_.size() < (int64_t)e->pages.size()) {
             err = "kv_evict: host tier is full or absent";
@@ -247,9 +342,11 @@ int KvPool::evict(uint64_t user, bool spill, void *side, std::string &err)
         }
         std::vector<int32_t> hp;
         for (size_t i = 0; i < e->pages.size(); ++i) { hp.push_back(free_host_.back()); free_host_.pop_back(); }
-        // the copy runs after the producer and after the last enqueued reader of these pages
-        int rc = wait_ticket(side, e->last_use_ticket);
-        if (rc == 0) rc = wait_ticket(side, e->ready_ticket);
+        // the copy runs after the producer and every enqueued reader of these pages, and after whatever may still be
+        // writing the host pages it lands in
+        int rc = 0;
+        for (int64_t t : release_after) if (rc == 0) rc = wait_ticket(side, t);
+        if (rc == 0) rc = wait_host_pages_released(side, hp);
         if (rc == 0) rc = copy_pages(true, e->pages, hp, side);
         const int64_t t = rc == 0 ? new_ticket(side) : -2;
         if (rc != 0 || t == -2) {
@@ -259,7 +356,7 @@ int KvPool::evict(uint64_t user, bool spill, void *side, std::string &err)
         }
         e->host_pages.swap(hp);
         e->host_ticket = t;
-        release_after = t;
+        release_after.assign(1, t);                   // recorded behind everything the copy waited for
         st_.spills += 1;
         st_.spill_bytes += (int64_t)(e->host_pages.size() * page_bytes_);
     }
@@ -268,7 +365,8 @@ int KvPool::evict(uint64_t user, bool spill, void *side, std::string &err)
         users_.erase(user);
     } else {
         e->state = UserState::Host;
-        e->ready_ticket = e->last_use_ticket = -1;
+        e->ready_ticket = -1;
+        e->use_tickets.clear();
     }
     return 0;
 }
@@ -296,12 +394,18 @@ int KvPool::reload(uint64_t user, void *side, void **ready_out, std::string &err
     if (rc == 0) rc = copy_pages(false, pages, e->host_pages, side);
     const int64_t t = rc == 0 ? new_ticket(side) : -2;
     if (rc != 0 || t == -2) {
-        release_pages(pages, -1);
+        // the user stays in HOST; the pages go back, still behind whatever their earlier owners left pending, and behind
+        // the part of this reload that may have been enqueued
+        std::vector<int64_t> behind;
+        const int64_t tf = new_ticket(side);
+        if (tf >= 0) behind.push_back(tf);
+        release_pages(pages, behind);
         err = "kv_reload: copy could not be enqueued";
         return RELAYGR_E_CUDA;
     }
     e->pages.swap(pages);
-    e->ready_ticket = e->last_use_ticket = t;
+    e->ready_ticket = t;
+    e->use_tickets.clear();
     e->state = UserState::Loading;
     st_.reloads += 1;
     st_.reload_bytes += (int64_t)(e->pages.size() * page_bytes_);

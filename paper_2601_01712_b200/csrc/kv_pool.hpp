@@ -26,6 +26,8 @@ struct Backend {
     virtual int event_record(void *ev, void *stream) = 0;
     virtual bool event_done(void *ev) = 0;
     virtual int stream_wait(void *stream, void *ev) = 0;
+    // Test control (host backend only; see relaygr_kv_host_backend_control).  Returns a negative status when unsupported.
+    virtual int64_t control(int32_t what, int64_t arg) { (void)what; (void)arg; return RELAYGR_E_UNSUPPORTED; }
 };
 
 Backend *make_cuda_backend();
@@ -38,8 +40,8 @@ struct UserEntry {
     int32_t prefix_len;
     std::vector<int32_t> pages;       // HBM page ids, logical order (empty when Host)
     std::vector<int32_t> host_pages;  // host-tier page ids (empty when no host copy)
-    int64_t ready_ticket = -1;        // producer of the HBM copy (pre-infer or reload)
-    int64_t last_use_ticket = -1;     // last enqueued reader / writer of the HBM pages
+    int64_t ready_ticket = -1;        // producer of the HBM copy (pre-infer, commit or reload)
+    std::vector<int64_t> use_tickets; // enqueued readers of the HBM pages that may still be running (any stream)
     int64_t host_ticket = -1;         // spill copy that fills the host pages
 };
 
@@ -73,16 +75,22 @@ public:
     int32_t tier_of(UserEntry &e);
 
     // Ordering helpers used by the compute calls.
-    int64_t new_ticket(void *stream);                  // records an event on stream; -1 on failure
+    int64_t new_ticket(void *stream);                  // records an event on stream; -2 on failure
     bool ticket_done(int64_t t);
     void *ticket_event(int64_t t);                     // nullptr when done / unknown
     int wait_ticket(void *stream, int64_t t);          // make stream wait for t (no-op if done)
     int wait_pages_released(void *stream, const std::vector<int32_t> &pages);
+    void add_use(UserEntry &e, int64_t ticket);        // remember a reader of the user's HBM pages
+    int wait_pages_of(uint64_t user, void *stream, std::string &err);
     void count_hit(int32_t tier);
 
 private:
     int take_pages(int32_t n, const int32_t *ids, std::vector<int32_t> &out, std::string &err);
-    void release_pages(std::vector<int32_t> &pages, int64_t ticket);
+    // Every ticket that must complete before the user's HBM pages may be overwritten: producer, readers, spill copy.
+    std::vector<int64_t> pending_of(UserEntry &e);
+    void release_pages(std::vector<int32_t> &pages, const std::vector<int64_t> &behind);
+    void release_host_pages(std::vector<int32_t> &pages, int64_t behind);
+    int wait_host_pages_released(void *stream, const std::vector<int32_t> &pages);
     void trim_tickets();
     int copy_pages(bool to_host, const std::vector<int32_t> &dev, const std::vector<int32_t> &host, void *stream);
 
@@ -93,7 +101,10 @@ private:
     int64_t n_pages_, n_host_pages_;
     std::vector<int32_t> free_pages_, free_host_;
     std::vector<uint8_t> page_used_;
-    std::vector<int64_t> page_release_ticket_;        // per HBM page: reuse only behind this ticket
+    // per HBM page: reuse only behind ALL of these tickets (a page may change hands while the copy or the kernels of an
+    // earlier owner are still running, so one ticket per page is not enough)
+    std::vector<std::vector<int64_t>> page_release_;
+    std::vector<int64_t> host_release_;               // per host page: the spill copy that may still be writing it
     std::unordered_map<uint64_t, UserEntry> users_;
     std::deque<Ticket> tickets_;
     int64_t ticket_base_ = 0;

@@ -235,7 +235,26 @@ int32_t relaygr_kv_commit(relaygr_kv_pool *pool, uint64_t user, void *stream)
     const int64_t t = kp.new_ticket(stream);
     if (t == -2) return fail(RELAYGR_E_CUDA, "kv_commit: could not record event");
     e->state = UserState::Resident;
-    e->ready_ticket = e->last_use_ticket = t;
+    e->ready_ticket = t;
+    e->use_tickets.clear();
+    return RELAYGR_OK;
+}
+
+int32_t relaygr_kv_wait_pages(relaygr_kv_pool *pool, uint64_t user, void *stream)
+{
+    if (!pool) return fail(RELAYGR_E_INVALID, "pool is NULL");
+    std::string err;
+    const int rc = pool->pool->wait_pages_of(user, stream, err);
+    return rc ? fail(rc, err) : rc;
+}
+
+int32_t relaygr_kv_host_backend_control(relaygr_kv_pool *pool, int32_t what, int64_t arg, int64_t *out)
+{
+    if (!pool) return fail(RELAYGR_E_INVALID, "pool is NULL");
+    const int64_t r = pool->be->control(what, arg);
+    if (r < 0) return fail((int)r, r == RELAYGR_E_UNSUPPORTED ? "host_backend_control: only pools of a host-only context have a controllable backend"
+                                                               : "host_backend_control: unknown request");
+    if (out) *out = r;
     return RELAYGR_OK;
 }
 
@@ -366,7 +385,7 @@ int32_t relaygr_preinfer(relaygr_ctx *ctx, relaygr_kv_pool *pool, int32_t n_user
     if (rc) return rc;
     const int64_t t = kp.new_ticket(stream);
     if (t == -2) return fail(RELAYGR_E_CUDA, "preinfer: could not record completion event");
-    for (UserEntry *e : entries) { e->state = UserState::Resident; e->ready_ticket = e->last_use_ticket = t; }
+    for (UserEntry *e : entries) { e->state = UserState::Resident; e->ready_ticket = t; e->use_tickets.clear(); }
     return RELAYGR_OK;
 }
 
@@ -400,6 +419,7 @@ int32_t relaygr_rank(relaygr_ctx *ctx, relaygr_kv_pool *pool, int32_t n_users, c
 
     CallDesc call;
     call.mode = MODE_RANK;
+    if ((int64_t)short_off[n_users] + (int64_t)cand_off[n_users] > 0x7fffffff) return fail(RELAYGR_E_UNSUPPORTED, "more than 2^31 rows in one call");
     int32_t row = 0;
     for (int i = 0; i < n_users; ++i) {
         const int P = entries[(size_t)i]->prefix_len;
@@ -428,7 +448,7 @@ int32_t relaygr_rank(relaygr_ctx *ctx, relaygr_kv_pool *pool, int32_t n_users, c
     if (rc) return rc;
     const int64_t t = kp.new_ticket(stream);
     if (t == -2) return fail(RELAYGR_E_CUDA, "rank: could not record completion event");
-    for (UserEntry *e : entries) e->last_use_ticket = t;
+    for (UserEntry *e : entries) kp.add_use(*e, t);      // every reader counts: several ctx may rank one user on different streams
     return RELAYGR_OK;
 }
 

@@ -243,3 +243,129 @@ def test_lookup_counts_hits_by_tier():
     B.relaygr_kv_lookup(hp.pool, 1)
     st = B.relaygr_kv_stats(hp.pool)
     assert (st["hits_hbm"], st["hits_host"], st["misses"]) == (1, 1, 1)
+
+
+# ---------------------------------------------------------------- states that need time on a GPU (Section 3.4), held by hand
+def _ctl(hp, what, arg=0):
+    return B.relaygr_kv_host_backend_control(hp.pool, what, arg)[1]
+
+
+def _resident(hp, user, prefix_len, fill):
+    _make_resident(hp, user, prefix_len, fill)
+    B.relaygr_kv_commit(hp.pool, user)
+
+
+def test_loading_state_busy_codes_and_promotion():
+    """A reload in flight: LOADING, single-flight, E_BUSY on evict / free, HBM once its event completes."""
+    hp = HostPool(4, 8)
+    _resident(hp, 1, 128, 5)
+    want = _content(hp, 1)
+    B.relaygr_kv_evict(hp.pool, 1, 1)
+    hp.hbm[:] = 0
+    _ctl(hp, B.HOSTCTL_MANUAL_EVENTS, 1)
+    code, ev = B.relaygr_kv_reload_from_host(hp.pool, 1)
+    assert code == B.OK and ev is not None
+    assert B.relaygr_kv_lookup(hp.pool, 1)[0] == B.TIER_LOADING
+    code2, ev2 = B.relaygr_kv_reload_from_host(hp.pool, 1)          # single-flight: the same event, nothing new enqueued
+    assert code2 == B.OK and ev2 == ev and B.relaygr_kv_stats(hp.pool)["reloads"] == 1
+    assert B.relaygr_kv_evict(hp.pool, 1, 1, ok=(B.E_BUSY,)) == B.E_BUSY
+    assert B.relaygr_kv_evict(hp.pool, 1, 0, ok=(B.E_BUSY,)) == B.E_BUSY
+    assert B.relaygr_kv_free(hp.pool, 1, ok=(B.E_BUSY,)) == B.E_BUSY
+    st = B.relaygr_kv_stats(hp.pool)
+    assert st["users_loading"] == 1 and st["users_hbm"] == 0
+    assert _ctl(hp, B.HOSTCTL_COMPLETE_EVENTS, -1) >= 1
+    assert B.relaygr_kv_lookup(hp.pool, 1)[0] == B.TIER_HBM
+    assert B.relaygr_kv_reload_from_host(hp.pool, 1) == (B.OK, None)
+    assert all(np.array_equal(a, b) for a, b in zip(_content(hp, 1), want))
+    B.relaygr_kv_evict(hp.pool, 1, 0)                                # allowed again
+    assert B.relaygr_kv_lookup(hp.pool, 1)[0] == B.TIER_HOST
+
+
+def test_bounded_number_of_reloads_in_flight():
+    """Section 3.4: reloads are rate-limited; beyond the bound the probe reports E_BUSY and the user stays in DRAM."""
+    hp = HostPool(8, 8)
+    for u in (1, 2, 3):
+        _resident(hp, u, 64, u)
+        B.relaygr_kv_evict(hp.pool, u, 1)
+    B.relaygr_kv_set_max_inflight_reloads(hp.pool, 2)
+    _ctl(hp, B.HOSTCTL_MANUAL_EVENTS, 1)
+    assert B.relaygr_kv_reload_from_host(hp.pool, 1)[0] == B.OK
+    assert B.relaygr_kv_reload_from_host(hp.pool, 2)[0] == B.OK
+    code, ev = B.relaygr_kv_reload_from_host(hp.pool, 3, ok=(B.E_BUSY,))
+    assert code == B.E_BUSY and ev is None
+    assert B.relaygr_kv_lookup(hp.pool, 3)[0] == B.TIER_HOST
+    assert B.relaygr_kv_stats(hp.pool)["pages_free"] == 6            # the refused reload took no pages
+    assert _ctl(hp, B.HOSTCTL_COMPLETE_EVENTS, 1) == 1               # the oldest reload lands
+    assert B.relaygr_kv_reload_from_host(hp.pool, 3)[0] == B.OK
+    assert B.relaygr_kv_stats(hp.pool)["reloads"] == 3
+
+
+def test_failed_reload_leaves_the_user_in_dram_with_its_pages_returned():
+    hp = HostPool(4, 8)
+    _resident(hp, 1, 128, 9)
+    want = _content(hp, 1)
+    B.relaygr_kv_evict(hp.pool, 1, 1)
+    _ctl(hp, B.HOSTCTL_FAIL_COPIES, 1)
+    code, ev = B.relaygr_kv_reload_from_host(hp.pool, 1, ok=(B.E_CUDA,))
+    assert code == B.E_CUDA and ev is None
+    assert B.relaygr_kv_lookup(hp.pool, 1) == (B.TIER_HOST, 128)
+    st = B.relaygr_kv_stats(hp.pool)
+    assert st["pages_free"] == 4 and st["reloads"] == 0 and st["host_pages_free"] == 6
+    hp.hbm[:] = 0
+    assert B.relaygr_kv_reload_from_host(hp.pool, 1)[0] == B.OK      # the next probe succeeds
+    assert all(np.array_equal(a, b) for a, b in zip(_content(hp, 1), want))
+
+
+def test_failed_spill_changes_nothing():
+    hp = HostPool(4, 8)
+    _resident(hp, 1, 128, 9)
+    _ctl(hp, B.HOSTCTL_FAIL_COPIES, 1)
+    assert B.relaygr_kv_evict(hp.pool, 1, 1, ok=(B.E_CUDA,)) == B.E_CUDA
+    assert B.relaygr_kv_lookup(hp.pool, 1)[0] == B.TIER_HBM
+    st = B.relaygr_kv_stats(hp.pool)
+    assert st["host_pages_free"] == 8 and st["pages_free"] == 2 and st["spills"] == 0
+
+
+def test_pages_stay_behind_an_earlier_owners_spill_when_they_change_hands_twice():
+    """User A's spill copy is still running when its pages go to B, who gives them back without using them; the next
+    owner must still wait for A's copy (a page remembers every pending ticket, not only the last owner's)."""
+    hp = HostPool(2, 8)
+    _resident(hp, 1, 64, 1)                                          # A: page 0
+    _resident(hp, 3, 64, 3)                                          # C: page 1
+    B.relaygr_kv_evict(hp.pool, 3, 1)                                # C's spill completes at once
+    _ctl(hp, B.HOSTCTL_MANUAL_EVENTS, 1)
+    B.relaygr_kv_evict(hp.pool, 1, 1)                                # A's spill stays pending
+    assert _ctl(hp, B.HOSTCTL_PENDING_EVENTS) == 1
+    a_page = 0
+    B.relaygr_kv_alloc(hp.pool, 2, 64, [a_page])                     # B takes A's page ...
+    B.relaygr_kv_free(hp.pool, 2)                                    # ... and returns it unused
+    B.relaygr_kv_alloc(hp.pool, 4, 64, [1])                          # keep the other page busy
+    waits0 = _ctl(hp, B.HOSTCTL_STREAM_WAITS)
+    assert B.relaygr_kv_reload_from_host(hp.pool, 3)[0] == B.OK      # C reloads into A's old page
+    assert list(B.relaygr_kv_pages(hp.pool, 3)) == [a_page]
+    assert _ctl(hp, B.HOSTCTL_STREAM_WAITS) == waits0 + 1            # behind A's pending spill copy
+    # relaygr_kv_wait_pages makes the same wait available to a caller that fills pages itself
+    _ctl(hp, B.HOSTCTL_COMPLETE_EVENTS, -1)
+    B.relaygr_kv_evict(hp.pool, 3, 0)
+    B.relaygr_kv_alloc(hp.pool, 5, 64, [a_page])
+    waits1 = _ctl(hp, B.HOSTCTL_STREAM_WAITS)
+    B.relaygr_kv_wait_pages(hp.pool, 5)
+    assert _ctl(hp, B.HOSTCTL_STREAM_WAITS) == waits1                # everything has completed: nothing to wait for
+    assert B.relaygr_kv_wait_pages(hp.pool, 77, ok=(B.E_MISS,)) == B.E_MISS
+
+
+def test_host_pages_stay_behind_a_pending_spill_when_their_user_is_freed():
+    hp = HostPool(4, 1)
+    _resident(hp, 1, 64, 1)
+    _resident(hp, 2, 64, 2)
+    _ctl(hp, B.HOSTCTL_MANUAL_EVENTS, 1)
+    B.relaygr_kv_evict(hp.pool, 1, 1)                                # spill of user 1 into the only host page: pending
+    B.relaygr_kv_free(hp.pool, 1)                                    # the host page is free again, the copy is not done
+    waits0 = _ctl(hp, B.HOSTCTL_STREAM_WAITS)
+    B.relaygr_kv_evict(hp.pool, 2, 1)                                # user 2 spills into the same host page
+    assert _ctl(hp, B.HOSTCTL_STREAM_WAITS) >= waits0 + 1
+
+
+def test_host_backend_control_is_refused_for_unknown_requests():
+    hp = HostPool(2, 0)
+    assert B.relaygr_kv_host_backend_control(hp.pool, 99, 0, ok=(B.E_INVALID,))[0] == B.E_INVALID
