@@ -4,7 +4,9 @@
 One step = one ``relaygr_rank`` call over a batch of the production-shaped workload
 (32 users x 2048-token prefix already pre-inferred into the paged pool, 64 short-term
 tokens, 512 candidates per user).  The prefix pre-infer and the full recompute of the
-same batch are timed beside it and reported in the same JSON line.  Prints ONE JSON line.
+same batch are timed beside it.  On one GPU the same line also carries the long-prefix
+workload (8 layers, d_model 512; 8192- and 24576-token prefixes), the reload-tier workload
+(DRAM tier behind the HBM pool) and single-request latencies.  Prints ONE JSON line.
 
     python bench.py --gpus 1 --steps 500 --warmup 20
     python -m torch.distributed.run --nproc-per-node N ... bench.py --gpus N ...   (N independent replicas)
@@ -29,22 +31,36 @@ METRIC = "candidates ranked/s with cached prefix KV (rank on cache); p50/p99 ran
 UNIT = "candidates/s"
 WORKLOAD = "config2: 4 layers, d_model 256, 4 heads x 64, FFN 1024, bf16; 32 users x (prefix 2048 cached, 64 short-term, 512 candidates); Zipf(1.1) ids over 1M items"
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of this workload's rank step, from the ncu captures
-# summarised under profiles/ (None = no capture of the kernel as it stands).
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the config-2 rank step, from the ncu captures summarised
+# under profiles/ (None = no capture of the kernel as it stands).
 DRAM_TRAFFIC_BYTES = {"attention": 121.2e6, "gemm": 19.7e6}      # gemm: mean of QKV (9.9 MB) and the fused out-proj + feed-forward kernel (29.6 MB)
+
+MIN_RANK_CALLS, MIN_FULL_CALLS = 500, 100       # individually timed calls behind every p50 / p99 of the main workload
 
 
 def load_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
         p = json.load(open(path))
-        return {"hbm_gbs": p["hbm_gbs"], "tflops": p.get("bf16_tflops_sustained", p["bf16_tflops"]),
-                "tflops_burst": p["bf16_tflops"], "source": "measured (MEASURED_PEAKS.json, sustained bf16)"}
-    return {"hbm_gbs": 6650.0, "tflops": 1400.0, "tflops_burst": 1590.0, "source": "fallback (earlier pool measurement)"}
+        return {"hbm_gbs": p["hbm_gbs"], "tflops_sustained": p.get("bf16_tflops_sustained", p["bf16_tflops"]),
+                "tflops_burst": p["bf16_tflops"], "sustained_mhz": (p.get("clocks_under_load") or {}).get("sm_mhz_median"),
+                "source": "measured (MEASURED_PEAKS.json)"}
+    return {"hbm_gbs": 6650.0, "tflops_sustained": 1400.0, "tflops_burst": 1590.0, "sustained_mhz": 1300.0,
+            "source": "fallback (earlier pool measurement)"}
+
+
+def fractions(tflops, clocks, peaks):
+    """A rate against both measured peaks.  The headline fraction takes the peak that was measured at the clock this leg
+    ran at: the burst figure when the sampled SM clock stayed near its maximum, the sustained one when the power cap pulled it down."""
+    sm, mx = (clocks or {}).get("sm_mhz"), (clocks or {}).get("sm_max_mhz")
+    capped = bool(sm and mx and sm < 0.93 * mx)
+    which = "sustained" if capped else "burst"
+    return {"tflops": tflops, "frac_burst": tflops / peaks["tflops_burst"], "frac_sustained": tflops / peaks["tflops_sustained"],
+            "frac": tflops / peaks["tflops_" + which], "headline_peak": which, "sm_mhz": sm}
 
 
 class ClockSampler:
-    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    """Samples SM clocks and throttle reasons with nvidia-smi while a timed region runs."""
     Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
          "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
@@ -60,6 +76,7 @@ class ClockSampler:
             self.thread.start()
         except Exception:
             self.proc = None
+        return self
 
     def count(self):
         return len(self.rows) if self.proc else 1 << 30
@@ -122,6 +139,97 @@ def reference_arm(args):
         "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
 
 
+# ---------------------------------------------------------------------------------------------------------------------
+# timing helpers (CUDA events on the launching stream)
+# ---------------------------------------------------------------------------------------------------------------------
+def timed_calls(torch, stream, fn, n, warmup=0):
+    """n calls of fn(i), each timed by itself with the stream idle before it (per-call latency as a request sees it).
+    Returns (device ms per call, host microseconds spent inside fn per call)."""
+    for i in range(warmup):
+        fn(i)
+    ms, host_us = [], []
+    for i in range(n):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record(stream)
+        t0 = time.perf_counter()
+        fn(i)
+        host_us.append((time.perf_counter() - t0) * 1e6)
+        e1.record(stream)
+        e1.synchronize()
+        ms.append(e0.elapsed_time(e1))
+    return np.array(ms), np.array(host_us)
+
+
+def pct(a):
+    return {"p50": float(np.percentile(a, 50)), "p99": float(np.percentile(a, 99)), "mean": float(np.mean(a)), "n": int(len(a))}
+
+
+def preinfer_ms(torch, stream, workloads, built, n, warmup=3):
+    pool = built.pool
+    pool.preinfer(built.dev_batches[0])
+    for _ in range(warmup):
+        workloads.realloc_users(built)
+        pool.preinfer(built.dev_batches[0])
+    torch.cuda.synchronize()
+    out = []
+    for _ in range(n):
+        workloads.realloc_users(built)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        pool.preinfer(built.dev_batches[0])
+        e1.record(stream)
+        e1.synchronize()
+        out.append(e0.elapsed_time(e1))
+    return np.array(out)
+
+
+def workload_leg(torch, workloads, shape, peaks, local, model, seed, p_lens, s_lens, c_lens, n_rank, n_full, n_pre, name):
+    """Pre-infer, rank on cache and full recompute of one batch, each with its own clock record and roofline fractions."""
+    built = workloads.build(shape, seed, p_lens, s_lens, c_lens, n_rotations=4, model=model)
+    pool, stream = built.pool, torch.cuda.current_stream()
+    b0 = built.batches[0]
+    n_cand = int(sum(c_lens))
+    scores = torch.empty(max(1, n_cand), dtype=torch.float32, device=model.device)
+    nrot = len(built.dev_batches)
+    out = {"workload": name, "users": len(p_lens), "prefix_tokens": int(sum(p_lens)), "candidates": n_cand}
+
+    sampler = ClockSampler(local).start()
+    pre = preinfer_ms(torch, stream, workloads, built, n_pre)
+    clocks = sampler.stop()
+    pre_ms = float(np.median(pre))
+    out["preinfer"] = {"ms": pre_ms, "tokens_per_s": int(sum(p_lens)) / (pre_ms * 1e-3), "n": int(len(pre)), "clocks": clocks,
+                       **fractions(workloads.batch_flops(shape, b0, "preinfer") / (pre_ms * 1e-3) / 1e12, clocks, peaks)}
+
+    sampler = ClockSampler(local).start()
+    lat, host = timed_calls(torch, stream, lambda i: pool.rank(built.dev_batches[i % nrot], scores), n_rank, warmup=5)
+    clocks = sampler.stop()
+    rank_ms = float(np.median(lat))
+    out["rank"] = {"ms": rank_ms, "latency_ms": pct(lat), "candidates_per_s": n_cand / (rank_ms * 1e-3), "host_us_per_call": float(np.median(host)),
+                   "clocks": clocks, **fractions(workloads.batch_flops(shape, b0, "rank") / (rank_ms * 1e-3) / 1e12, clocks, peaks)}
+
+    sampler = ClockSampler(local).start()
+    flat, _ = timed_calls(torch, stream, lambda i: model.rank_full(built.dev_batches[i % nrot], scores), n_full, warmup=2)
+    clocks = sampler.stop()
+    full_ms = float(np.median(flat))
+    out["full_recompute"] = {"ms": full_ms, "latency_ms": pct(flat), "clocks": clocks,
+                             **fractions(workloads.batch_flops(shape, b0, "full") / (full_ms * 1e-3) / 1e12, clocks, peaks)}
+    out["rank_beats_full_recompute_p99"] = bool(np.percentile(lat, 99) < np.percentile(flat, 99))
+    assert model.device_status() == 0, "a kernel reported an internal error"
+    built.pool.close()
+    del built, scores
+    torch.cuda.empty_cache()
+    return out
+
+
+def guarded(fn):
+    """A leg that fails must not cost the line: its error is reported in its place."""
+    try:
+        return fn()
+    except Exception as e:      # noqa: BLE001
+        return {"error": "%s: %s" % (type(e).__name__, str(e)[:300])}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -129,6 +237,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-legs", action="store_true", help="only the metric's own workload (no long-prefix, reload-tier and single-request legs)")
+    ap.add_argument("--tier-population", type=int, default=4096, help="users of the reload-tier leg (their K/V sits in pinned DRAM; 16 MiB each)")
     ap.add_argument("--workload", type=int, default=2, choices=[2, 3, 4],
                     help="2 = production-shaped rank (the metric's workload), 3 = jagged batch with shuffled pages, 4 = long-sequence model")
     ap.add_argument("--users", type=int, default=0, help="0 = the workload's own batch size")
@@ -138,6 +248,7 @@ def main():
     ap.add_argument("--d-model", type=int, default=0, help="override the model's width (heads of 64, FFN 4x; sweeps)")
     ap.add_argument("--attention", default="softmax", choices=["softmax", "pointwise"],
                     help="pointwise: the HSTU-style SiLU attention variant of the same model (sweeps)")
+    ap.add_argument("--dtype", default="bf16", choices=["bf16", "f32"], help="f32: the fp32 model and fp32 K/V pages (CUDA-core kernels; sweeps)")
     args = ap.parse_args()
     if args.impl == "reference":
         return reference_arm(args)
@@ -162,12 +273,14 @@ def main():
     wl = synth.workload(args.workload)
     shape = wl.model
     pointwise = args.attention == "pointwise"
-    if args.layers or args.d_model or pointwise:
+    f32 = args.dtype == "f32"
+    if args.layers or args.d_model or pointwise or f32:
         dm = args.d_model or shape.d_model
-        shape = synth.ModelShape(args.layers or shape.n_layers, dm, dm // 64, 64, 4 * dm, shape.vocab, shape.dtype,
+        shape = synth.ModelShape(args.layers or shape.n_layers, dm, dm // 64, 64, 4 * dm, shape.vocab, synth.DTYPE_F32 if f32 else shape.dtype,
                                  attn_kind=1 if pointwise else 0)
-    custom = ("; overrides: layers %d, d_model %d%s" % (shape.n_layers, shape.d_model, ", pointwise SiLU attention" if pointwise else "")) \
-        if (args.layers or args.d_model or pointwise) else ""
+    custom = ("; overrides: layers %d, d_model %d%s%s" % (shape.n_layers, shape.d_model, ", pointwise SiLU attention" if pointwise else "",
+                                                          ", fp32 model and fp32 K/V pages" if f32 else "")) \
+        if (args.layers or args.d_model or pointwise or f32) else ""
     if args.workload == 3:
         n_users = args.users or 128
         pl, sl, cl = synth.config3_lengths(np.random.default_rng(wl.seed + 1000 * rank), n_users)
@@ -184,13 +297,19 @@ def main():
         p_lens, s_lens, c_lens = [P] * n_users, [64] * n_users, [C] * n_users
         workload_name = WORKLOAD if (n_users, P, C, custom) == (32, 2048, 512, "") else \
             "config2 model; %d users x (prefix %d cached, 64 short-term, %d candidates)%s" % (n_users, P, C, custom)
-    # replicas: every rank holds its own users (user-hash placement), no data-path collective
+    # replicas: every rank holds the users that hash to it (affinity routing by user id), no data-path collective
+    user_ids, u = [], 0
+    while len(user_ids) < n_users:
+        if replicas.owner_rank(u, world) == rank:
+            user_ids.append(u)
+        u += 1
     built = workloads.build(shape, wl.seed + 1000 * rank, p_lens, s_lens, c_lens, n_rotations=8, shuffle_pages=args.workload == 3,
-                            first_user=rank * n_users, device="cuda:%d" % local)
+                            user_ids=user_ids, device="cuda:%d" % local)
     model, pool = built.model, built.pool
     stream = torch.cuda.current_stream()
     n_cand = int(sum(c_lens))
     scores = torch.empty(n_cand, dtype=torch.float32, device=model.device)
+    peaks = load_peaks()
 
     def barrier():
         if dist is not None:
@@ -201,21 +320,10 @@ def main():
         return replicas.max_over_ranks(ms, dist, model.device)
 
     # ---- pre-infer (timed beside the metric) --------------------------------------------------------
-    pre_steps = max(3, min(20, args.steps // 20))
-    pool.preinfer(built.dev_batches[0])
-    for _ in range(3):
-        workloads.realloc_users(built)
-        pool.preinfer(built.dev_batches[0])
-    torch.cuda.synchronize()
-    pre_ms = []
-    for _ in range(pre_steps):
-        workloads.realloc_users(built)
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(stream)
-        pool.preinfer(built.dev_batches[0])
-        e1.record(stream)
-        e1.synchronize()
-        pre_ms.append(e0.elapsed_time(e1))
+    pre_steps = max(20, min(40, args.steps // 10)) if sum(p_lens) < 200_000 else max(3, min(20, args.steps // 20))
+    sampler = ClockSampler(local).start()
+    pre_ms = preinfer_ms(torch, stream, workloads, built, pre_steps)
+    pre_clocks = sampler.stop()
     pre_ms_med = float(np.median(pre_ms))
     # per-kernel-class timing of pre-infer (events around every launch; separate from the timing above)
     B.relaygr_profile_enable(model.ctx, True)
@@ -241,6 +349,7 @@ def main():
         evs[i + 1].record(stream)
     barrier()
     torch.cuda.synchronize()
+    launches = model.launch_count() - launches0
     # a timed region shorter than a few sampling periods: keep the same load running (untimed) until the sampler has seen it
     extra = 0
     while sampler.count() < 3 and extra < 20000:
@@ -252,37 +361,17 @@ def main():
     clocks = sampler.stop()
     total_ms = max_over_ranks(evs[0].elapsed_time(evs[-1]))
     lat = np.array([evs[i].elapsed_time(evs[i + 1]) for i in range(args.steps)])
-    launches = model.launch_count() - launches0
     assert model.device_status() == 0, "a kernel reported an internal error"
     ms_per_step = total_ms / args.steps
     value = world * n_cand / (ms_per_step * 1e-3)
 
-    # one call at a time (stream idle before each call): per-call latency as a request sees it
-    lat1 = []
-    for i in range(min(args.steps, 200)):
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        torch.cuda.synchronize()
-        e0.record(stream)
-        pool.rank(built.dev_batches[i % nrot], scores)
-        e1.record(stream)
-        e1.synchronize()
-        lat1.append(e0.elapsed_time(e1))
-    lat1 = np.array(lat1)
+    # one call at a time (stream idle before each call): per-call latency as a request sees it, and the host's share of it
+    n_lat = max(MIN_RANK_CALLS, min(args.steps, 2000)) if ms_per_step < 20 else max(100, min(args.steps, 500))
+    lat1, host_us = timed_calls(torch, stream, lambda i: pool.rank(built.dev_batches[i % nrot], scores), n_lat)
 
     # ---- full recompute of the same batches ---------------------------------------------------------
-    full_steps = max(5, min(100, args.steps // 5))
-    for i in range(3):
-        model.rank_full(built.dev_batches[i % nrot], scores)
-    torch.cuda.synchronize()
-    full_lat = []
-    for i in range(full_steps):
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(stream)
-        model.rank_full(built.dev_batches[i % nrot], scores)
-        e1.record(stream)
-        e1.synchronize()
-        full_lat.append(e0.elapsed_time(e1))
-    full_lat = np.array(full_lat)
+    n_full = MIN_FULL_CALLS if ms_per_step < 20 else 20
+    full_lat, _ = timed_calls(torch, stream, lambda i: model.rank_full(built.dev_batches[i % nrot], scores), n_full, warmup=3)
 
     # ---- per-kernel timing of the rank step (events around every launch; separate from the timed region)
     B.relaygr_profile_enable(model.ctx, True)
@@ -291,7 +380,6 @@ def main():
         pool.rank(built.dev_batches[i % nrot], scores)
     prof = B.relaygr_profile_read(model.ctx)
     B.relaygr_profile_enable(model.ctx, False)
-    peaks = load_peaks()
     prof_total = sum(prof[k] for k in prof if k.endswith("_ms"))
     b0 = built.batches[0]
     # algorithmic FLOPs of the two tensor-core kernel classes over one rank step (dead last-layer work excluded)
@@ -304,8 +392,11 @@ def main():
         ms = prof[cls + "_ms"] / n_launch                       # average launch duration, CUDA events on the launching stream
         fl = class_flops[cls] * prof_steps / n_launch           # algorithmic FLOPs per launch
         tf = fl / (ms * 1e-3) / 1e12
-        rooflines[cls] = {"kernel": class_name[cls], "bound": "tensor", "achieved": tf, "peak": peaks["tflops"], "unit": "TFLOP/s",
-                          "frac": tf / peaks["tflops"], "peak_source": peaks["source"], "traffic": DRAM_TRAFFIC_BYTES[cls] if workload_name == WORKLOAD else None,
+        fr = fractions(tf, clocks, peaks)
+        rooflines[cls] = {"kernel": class_name[cls], "bound": "tensor", "achieved": tf, "peak": peaks["tflops_" + fr["headline_peak"]], "unit": "TFLOP/s",
+                          "frac": fr["frac"], "frac_burst": fr["frac_burst"], "frac_sustained": fr["frac_sustained"],
+                          "peak_source": "%s, %s bf16 figure (median SM clock of the timed region %s MHz)" % (peaks["source"], fr["headline_peak"], fr["sm_mhz"]),
+                          "traffic": DRAM_TRAFFIC_BYTES[cls] if workload_name == WORKLOAD else None,
                           "ms_per_launch": ms, "launches_per_step": n_launch / prof_steps, "algorithmic_flops_per_launch": fl,
                           "share_of_step": prof[cls + "_ms"] / prof_total if prof_total else None}
     dominant = max(rooflines, key=lambda c: rooflines[c]["share_of_step"] or 0.0)
@@ -343,7 +434,7 @@ def main():
 
     # ---- CPU baseline: the checker, timed on this machine's host cores ----------------------------------
     cpu = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline and args.workload == 2:
+    if rank == 0 and world == 1 and not args.no_cpu_baseline and args.workload == 2 and not f32:
         from oracle import ref
         om = ref.Model(shape.n_layers, shape.d_model, shape.n_heads, shape.d_head, shape.d_ff, shape.ln_eps,
                        {**built.weights.mat, **built.weights.vec})
@@ -368,32 +459,87 @@ def main():
                          "(prefix K/V from the checker's own pre-infer, untimed); %.1f s of CPU work" % (n_sample, n_users, nrot, t_cpu),
                "max_abs_err_vs_gpu": err}
 
+    rank_flops = workloads.batch_flops(shape, b0, "rank")
+    pre_flops = workloads.batch_flops(shape, b0, "preinfer")
+    full_flops = workloads.batch_flops(shape, b0, "full")
+    full_med = float(np.median(full_lat))
+
+    # ---- further legs (one GPU, the metric's own workload only): single requests, long prefixes, the reload tier --------
+    legs = {}
+    if world == 1 and not args.no_legs and args.workload == 2 and not custom and (args.users, args.prefix, args.candidates) == (0, 0, 0):
+        def b1(model_, shape_, seed, P_, S_, C_, name):
+            return workload_leg(torch, workloads, shape_, peaks, local, model_, seed, [P_], [S_], [C_], MIN_RANK_CALLS, MIN_FULL_CALLS, 20, name)
+
+        legs["b1"] = {"config2": guarded(lambda: b1(model, shape, wl.seed + 7, 2048, 64, 512,
+                                                     "one request: config-2 model, one user (prefix 2048 cached, 64 short-term, 512 candidates)"))}
+        # the reload tier on the same model (its users' prefixes are 4096 tokens: 16 MiB of K/V each)
+        def tier():
+            from paper_2601_01712_b200 import tier_workload
+            last = None
+            for pop in (args.tier_population, args.tier_population // 2, args.tier_population // 4):      # the largest population the box can pin
+                try:
+                    rep = tier_workload.run(population=pop, hbm_users=pop // 4, calls=300, warmup=20, model=model)
+                    rep["population_tried_first"] = args.tier_population
+                    return rep
+                except RuntimeError as e:       # pinned allocation refused: halve
+                    last = e
+                    torch.cuda.empty_cache()
+            raise last
+        built.pool.close()
+        del built, pool
+        torch.cuda.empty_cache()
+        sampler = ClockSampler(local).start()
+        legs["tier"] = guarded(tier)
+        if isinstance(legs["tier"], dict):
+            legs["tier"]["clocks"] = sampler.stop()
+        model.close()
+        del model
+        torch.cuda.empty_cache()
+
+        def long_prefix():
+            from paper_2601_01712_b200 import runtime as rt
+            wl4 = synth.workload(4)
+            w4 = synth.make_weights(wl4.model, wl4.seed)
+            m4 = rt.Model(wl4.model, w4, "cuda:%d" % local)
+            del w4
+            out = {}
+            for P_, n_rank, n_full, n_pre in ((8192, 200, 20, 20), (24576, 100, 10, 20)):
+                out["P%d" % P_] = guarded(lambda: workload_leg(
+                    torch, workloads, wl4.model, peaks, local, m4, wl4.seed + P_, [P_] * 16, [128] * 16, [1024] * 16, n_rank, n_full, n_pre,
+                    "config4: 8 layers, d_model 512, 8 heads x 64, FFN 2048, bf16; 16 users x (prefix %d cached, 128 short-term, 1024 candidates)" % P_))
+            legs["b1"]["config4"] = guarded(lambda: workload_leg(
+                torch, workloads, wl4.model, peaks, local, m4, wl4.seed + 9, [8192], [128], [1024], MIN_RANK_CALLS, MIN_FULL_CALLS, 20,
+                "one request: config-4 model, one user (prefix 8192 cached, 128 short-term, 1024 candidates)"))
+            m4.close()
+            return out
+        legs["long_prefix"] = guarded(long_prefix)
+
     if rank == 0:
-        rank_flops = workloads.batch_flops(shape, b0, "rank")
-        pre_flops = workloads.batch_flops(shape, b0, "preinfer")
-        full_flops = workloads.batch_flops(shape, b0, "full")
+        rank_fr = fractions(rank_flops / (ms_per_step * 1e-3) / 1e12, clocks, peaks)
         out = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "bf16", "data": "synthetic",
+            "dtype": "f32" if f32 else "bf16", "data": "synthetic",
             "config": {"workload": workload_name, "step": "one relaygr_rank call over the batch, prefix KV already in the paged pool",
                        "users": n_users, "prefix_tokens": int(sum(p_lens)), "short_tokens": int(sum(s_lens)), "candidates": n_cand,
                        "l2": "inputs larger than L2: each step streams %.0f MiB of prefix K/V and rotates 8 input sets" % (shape.kv_bytes(int(sum(p_lens))) / 2**20),
-                       "parallelism": "replicas (users hashed to GPUs), no collective" if world > 1 else "single GPU"},
+                       "parallelism": "replicas (users placed by replicas.owner_rank(user id)), no collective" if world > 1 else "single GPU"},
             "latency_ms": {"rank_p50_backlogged": float(np.percentile(lat, 50)), "rank_p99_backlogged": float(np.percentile(lat, 99)),
-                           "rank_p50": float(np.percentile(lat1, 50)), "rank_p99": float(np.percentile(lat1, 99)),
+                           "rank_p50": float(np.percentile(lat1, 50)), "rank_p99": float(np.percentile(lat1, 99)), "rank_calls": int(len(lat1)),
                            "full_recompute_p50": float(np.percentile(full_lat, 50)), "full_recompute_p99": float(np.percentile(full_lat, 99)),
+                           "full_recompute_calls": int(len(full_lat)),
                            "rank_beats_full_recompute_p99": bool(np.percentile(lat1, 99) < np.percentile(full_lat, 99))},
-            "preinfer": {"tokens_per_s": int(sum(p_lens)) / (pre_ms_med * 1e-3), "ms": pre_ms_med,
-                         "frac_of_tensor_roofline": pre_flops / (pre_ms_med * 1e-3) / 1e12 / peaks["tflops"],
+            "host_us_per_rank_call": float(np.median(host_us)),
+            "preinfer": {"tokens_per_s": int(sum(p_lens)) / (pre_ms_med * 1e-3), "ms": pre_ms_med, "calls": int(len(pre_ms)), "clocks": pre_clocks,
+                         **fractions(pre_flops / (pre_ms_med * 1e-3) / 1e12, pre_clocks, peaks),
                          "kernel_ms": pre_kernel_ms},
-            "whole_step_roofline": {"rank_tflops": rank_flops / (ms_per_step * 1e-3) / 1e12,
-                                    "rank_frac": rank_flops / (ms_per_step * 1e-3) / 1e12 / peaks["tflops"],
-                                    "full_recompute_tflops": full_flops / (float(np.median(full_lat)) * 1e-3) / 1e12},
+            "whole_step_roofline": {"rank": rank_fr,
+                                    "full_recompute": fractions(full_flops / (full_med * 1e-3) / 1e12, clocks, peaks)},
             "roofline": rooflines[dominant], "roofline_second_kernel": rooflines[other],
             "kernel_ms_per_step": {k: prof[k] / prof_steps for k in prof if k.endswith("_ms")},
             "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks, "cpu_baseline": cpu,
         }
+        out.update(legs)
         print(json.dumps(out))
     if dist is not None:
         dist.destroy_process_group()

@@ -155,11 +155,16 @@ int32_t relaygr_set_workspace(relaygr_ctx *ctx, void *dev, size_t bytes);
 
 /*
  * Kernels never trap, and their internal waits are bounded: a kernel that meets an
- * impossible state (a wait that ran out) records a code in a status word at the start
- * of the workspace and the kernels after it return early, leaving results undefined.
- * This call SYNCHRONISES `stream`, then copies the word to *out (0 = healthy).
- * relaygr_set_workspace clears the word (synchronously).
+ * impossible state records a code in a status word at the start of the workspace - a
+ * wait that ran out (RELAYGR_DEVSTATUS_WAIT_TIMEOUT), a token id outside [0, vocab)
+ * (RELAYGR_DEVSTATUS_BAD_INDEX; a row that exists is read instead, so no access leaves
+ * the table).  The first code stays.  While the word is non-zero the tensor-core
+ * kernels of later calls return at once (results undefined, K/V pages not written), so
+ * an error cannot pile up.  This call SYNCHRONISES `stream`, then copies the word to
+ * *out (0 = healthy).  relaygr_set_workspace clears the word (synchronously).
  */
+#define RELAYGR_DEVSTATUS_WAIT_TIMEOUT 1
+#define RELAYGR_DEVSTATUS_BAD_INDEX    2
 int32_t relaygr_device_status(relaygr_ctx *ctx, void *stream, int32_t *out);
 
 /* ---- paged prefix-KV pool (Section 3.3 sliding window, Section 3.4 DRAM tier) ---------------- */
@@ -268,6 +273,8 @@ int32_t relaygr_kv_host_backend_control(relaygr_kv_pool *pool, int32_t what, int
 /*
  * The embedding gather alone (the first step of both passes): out[i, :] = emb[ids[i], :]
  * for n ids, a bit-exact row copy in cfg.dtype.  ids dev int32 [n], out dev [n, d].
+ * An id outside [0, vocab) is recorded as RELAYGR_DEVSTATUS_BAD_INDEX in the status word
+ * of the lent workspace (if one is lent).
  */
 int32_t relaygr_gather(relaygr_ctx *ctx, const int32_t *ids, int64_t n, void *out, void *stream);
 

@@ -15,6 +15,7 @@ LIB_PATH = os.path.join(_HERE, "librelaygr.so")
 OK, E_INVALID, E_NOSPACE, E_EXISTS, E_MISS, E_BUSY, E_CUDA, E_UNSUPPORTED = 0, -1, -2, -3, -4, -5, -6, -7
 DTYPE_F32, DTYPE_BF16 = 0, 1
 TIER_MISS, TIER_ALLOCATED, TIER_HBM, TIER_LOADING, TIER_HOST = 0, 1, 2, 3, 4
+DEVSTATUS_WAIT_TIMEOUT, DEVSTATUS_BAD_INDEX = 1, 2      # RELAYGR_DEVSTATUS_*: codes of the device status word
 
 STATUS_NAMES = {0: "OK", -1: "E_INVALID", -2: "E_NOSPACE", -3: "E_EXISTS", -4: "E_MISS", -5: "E_BUSY", -6: "E_CUDA",
                 -7: "E_UNSUPPORTED"}

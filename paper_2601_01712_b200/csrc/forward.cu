@@ -171,11 +171,12 @@ int Forward::upload(const std::vector<int32_t> &blob, size_t dst_off, cudaStream
 int Forward::gather(const int32_t *ids, int64_t n, void *out, cudaStream_t stream, std::string &err)
 {
     cudaError_t e;
+    int *status = (ws && ws_bytes >= 1024) ? reinterpret_cast<int *>(ws) : nullptr;      // the status word of the lent workspace, if any
     if (cfg.dtype == RELAYGR_DTYPE_F32)
-        e = launch_gather_rows<float>((const float *)w.emb, cfg.vocab, cfg.d_model, ids, n, (float *)out, stream, &launches);
+        e = launch_gather_rows<float>((const float *)w.emb, cfg.vocab, cfg.d_model, ids, n, (float *)out, status, stream, &launches);
     else
         e = launch_gather_rows<__nv_bfloat16>((const __nv_bfloat16 *)w.emb, cfg.vocab, cfg.d_model, ids, n, (__nv_bfloat16 *)out,
-                                              stream, &launches);
+                                              status, stream, &launches);
     if (e != cudaSuccess) { err = cuda_msg("gather", e); return RELAYGR_E_CUDA; }
     return RELAYGR_OK;
 }
@@ -340,7 +341,7 @@ int Forward::run_t(const CallDesc &call, float *scores, cudaStream_t stream, std
         const float *g1 = w.ln1_g + (size_t)l * d, *b1n = w.ln1_b + (size_t)l * d;
         if (l == 0) {
             cudaEvent_t pe = prof_begin(stream);
-            e = launch_gather_ln<T>((const T *)w.emb, cfg.vocab, d, src, R, g1, b1n, cfg.ln_eps, x, a, stream, &launches);
+            e = launch_gather_ln<T>((const T *)w.emb, cfg.vocab, d, src, R, g1, b1n, cfg.ln_eps, x, a, reinterpret_cast<int *>(ws + lay.status), stream, &launches);
             prof_end(KC_GATHER_LN, pe, stream);
         } else {
             e = layernorm(g1, b1n);

@@ -5,6 +5,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include "../../include/relaygr.h"
+
 namespace relaygr {
 
 // One user of a call.  Rows are the token rows the call computes (activations are
@@ -51,6 +53,10 @@ struct AttnMerge {
     int32_t seq, head, q0, n_q;
     int32_t slot0, n_splits;
 };
+
+// Codes a kernel may record in the status word at the start of the workspace (relaygr_device_status; 0 = healthy).
+// The first code recorded stays.
+enum DeviceStatus : int { STATUS_OK = 0, STATUS_WAIT_TIMEOUT = RELAYGR_DEVSTATUS_WAIT_TIMEOUT, STATUS_BAD_INDEX = RELAYGR_DEVSTATUS_BAD_INDEX };
 
 enum EpiMode : int32_t { EPI_STORE = 0, EPI_RESID = 1, EPI_QKV = 2 };
 

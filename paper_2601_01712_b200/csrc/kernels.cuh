@@ -44,15 +44,16 @@ struct PerDeviceValue {
 
 // ---- memory-bound steps (CUDA cores, vectorised loads, warp-shuffle reductions) ----------------
 
-// out[i, :] = emb[ids[i], :], a bit-exact row copy.
+// out[i, :] = emb[ids[i], :], a bit-exact row copy.  An id outside [0, vocab) records STATUS_BAD_INDEX in *err (err may
+// be nullptr) and row 0 / vocab - 1 is copied instead, so that no access leaves the table.
 template <typename T>
-cudaError_t launch_gather_rows(const T *emb, int64_t vocab, int d, const int32_t *ids, int64_t n, T *out,
+cudaError_t launch_gather_rows(const T *emb, int64_t vocab, int d, const int32_t *ids, int64_t n, T *out, int *err,
                                cudaStream_t stream, int64_t *launches);
 
 // x[r, :] = emb[id(r), :] widened to fp32 (the residual stream); a[r, :] = LN(x[r, :]; g, b) in T.
 template <typename T>
 cudaError_t launch_gather_ln(const T *emb, int64_t vocab, int d, RowSource src, int64_t n_rows,
-                             const float *g, const float *b, float eps, float *x, T *a,
+                             const float *g, const float *b, float eps, float *x, T *a, int *err,
                              cudaStream_t stream, int64_t *launches);
 
 // a[r, :] = LN(x[r, :]; g, b) in T.

@@ -50,13 +50,17 @@ __device__ __forceinline__ int row_token_id(const RowSource &src, int64_t row)
 
 template <typename T>
 __global__ void __launch_bounds__(kWarpsPerBlock * 32)
-gather_rows_kernel(const T *__restrict__ emb, int64_t vocab, int d, const int32_t *__restrict__ ids, int64_t n, T *__restrict__ out)
+gather_rows_kernel(const T *__restrict__ emb, int64_t vocab, int d, const int32_t *__restrict__ ids, int64_t n, T *__restrict__ out, int *err)
 {
     const int64_t row = (int64_t)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     if (row >= n) return;
     int64_t id = ids[row];
-    id = id < 0 ? 0 : (id >= vocab ? vocab - 1 : id);
+    if (id < 0 || id >= vocab) {
+        // an id outside the table: recorded in the status word (when there is one), and a row that exists is read instead
+        if (err && lane == 0) atomicCAS(err, (int)STATUS_OK, (int)STATUS_BAD_INDEX);
+        id = id < 0 ? 0 : vocab - 1;
+    }
     // 16-byte copies: d * sizeof(T) is a multiple of 16
     const int n16 = d * (int)sizeof(T) / 16;
     const uint4 *s = reinterpret_cast<const uint4 *>(emb + id * d);
@@ -114,7 +118,7 @@ __device__ __forceinline__ void ln_rows_store(const float4 (&v)[ROWS][NC], int d
 template <typename T, int NC, int ROWS>
 __global__ void __launch_bounds__(kWarpsPerBlock * 32)
 gather_ln_kernel(const T *__restrict__ emb, int64_t vocab, int d, RowSource src, int64_t n_rows,
-                 const float *__restrict__ g, const float *__restrict__ b, float eps, float *__restrict__ x, T *__restrict__ a)
+                 const float *__restrict__ g, const float *__restrict__ b, float eps, float *__restrict__ x, T *__restrict__ a, int *err)
 {
     grid_launch_dependents();
     grid_dependency_wait();
@@ -124,7 +128,11 @@ gather_ln_kernel(const T *__restrict__ emb, int64_t vocab, int d, RowSource src,
     long long my_id = 0;
     if (lane < ROWS && row0 + lane < n_rows) {
         my_id = row_token_id(src, row0 + lane);
-        my_id = my_id < 0 ? 0 : (my_id >= vocab ? vocab - 1 : my_id);
+        if (my_id < 0 || my_id >= vocab) {
+            // an id outside the table: recorded in the status word, and a row that exists is read instead
+            if (err) atomicCAS(err, (int)STATUS_OK, (int)STATUS_BAD_INDEX);
+            my_id = my_id < 0 ? 0 : vocab - 1;
+        }
     }
     float4 v[ROWS][NC];
 #pragma unroll
@@ -383,25 +391,25 @@ inline unsigned blocks_for(int64_t warps) { return (unsigned)((warps + kWarpsPer
 }  // namespace
 
 template <typename T>
-cudaError_t launch_gather_rows(const T *emb, int64_t vocab, int d, const int32_t *ids, int64_t n, T *out,
+cudaError_t launch_gather_rows(const T *emb, int64_t vocab, int d, const int32_t *ids, int64_t n, T *out, int *err,
                                cudaStream_t stream, int64_t *launches)
 {
     if (n == 0) return cudaSuccess;
-    gather_rows_kernel<T><<<blocks_for(n), kWarpsPerBlock * 32, 0, stream>>>(emb, vocab, d, ids, n, out);
+    gather_rows_kernel<T><<<blocks_for(n), kWarpsPerBlock * 32, 0, stream>>>(emb, vocab, d, ids, n, out, err);
     *launches += 1;
     return cudaGetLastError();
 }
 
 template <typename T>
 cudaError_t launch_gather_ln(const T *emb, int64_t vocab, int d, RowSource src, int64_t n_rows, const float *g,
-                             const float *b, float eps, float *x, T *a, cudaStream_t stream, int64_t *launches)
+                             const float *b, float eps, float *x, T *a, int *err, cudaStream_t stream, int64_t *launches)
 {
     if (n_rows == 0) return cudaSuccess;
     const int nc = (d + 127) / 128;
     cudaError_t e;
 #define RELAYGR_GLN(NC, ROWS)                                                                                             \
     e = launch_dependent(gather_ln_kernel<T, NC, ROWS>, dim3(blocks_for((n_rows + ROWS - 1) / ROWS)), dim3(kWarpsPerBlock * 32), 0, stream, 1, \
-                         emb, vocab, d, src, n_rows, g, b, eps, x, a)
+                         emb, vocab, d, src, n_rows, g, b, eps, x, a, err)
     if (nc <= 1) RELAYGR_GLN(1, 4);
     else if (nc <= 2) RELAYGR_GLN(2, 4);
     else if (nc <= 4) RELAYGR_GLN(4, 4);
@@ -480,9 +488,9 @@ cudaError_t launch_attention_simt(const T *q, const T *k_lin, const T *v_lin, Pa
 }
 
 #define RELAYGR_INSTANTIATE(T)                                                                                              \
-    template cudaError_t launch_gather_rows<T>(const T *, int64_t, int, const int32_t *, int64_t, T *, cudaStream_t, int64_t *); \
+    template cudaError_t launch_gather_rows<T>(const T *, int64_t, int, const int32_t *, int64_t, T *, int *, cudaStream_t, int64_t *); \
     template cudaError_t launch_gather_ln<T>(const T *, int64_t, int, RowSource, int64_t, const float *, const float *, float,  \
-                                             float *, T *, cudaStream_t, int64_t *);                                        \
+                                             float *, T *, int *, cudaStream_t, int64_t *);                                 \
     template cudaError_t launch_layernorm<T>(const float *, int, int64_t, const float *, const float *, float, T *,          \
                                              cudaStream_t, int64_t *);                                                      \
     template cudaError_t launch_gemm_simt<T>(const T *, const T *, int64_t, int, int, const Epilogue &, cudaStream_t,        \

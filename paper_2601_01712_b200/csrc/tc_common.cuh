@@ -14,7 +14,7 @@ namespace tc {
 
 constexpr long long kWaitLimitCycles = 2000000000LL;   // ~1 s at 2 GHz
 
-enum ErrCode : int { ERR_NONE = 0, ERR_WAIT_TIMEOUT = 1, ERR_BAD_INDEX = 2 };
+enum ErrCode : int { ERR_NONE = 0, ERR_WAIT_TIMEOUT = 1 };      // = RELAYGR_DEVSTATUS_WAIT_TIMEOUT of the public header
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 

@@ -118,7 +118,7 @@ class KvPool:
         self.slab = self._slab_raw[pad:pad + hbm_pages * pb]
         self.host = None
         if host_pages:
-            self.host = torch.empty(host_pages * pb, dtype=torch.uint8).pin_memory()
+            self.host = torch.empty(host_pages * pb, dtype=torch.uint8, pin_memory=True)     # allocated pinned, not copied into a pinned buffer
         self.pool = B.relaygr_kv_pool_create(model.ctx, self.slab.data_ptr(), self.slab.numel(),
                                              self.host.data_ptr() if self.host is not None else None,
                                              self.host.numel() if self.host is not None else 0)

@@ -37,20 +37,27 @@ class ZipfUsers:
 
 def run(population: int = 1024, hbm_users: int = 256, prefix: int = 4096, batch: int = 32, n_short: int = 64, n_cand: int = 512,
         calls: int = 300, warmup: int = 20, zipf_users: float = 0.9, seed: int = synth.BASE_SEED + 5, shape=None,
-        max_in_flight_calls: int = 2, device: str = "cuda:0", collect_scores: bool = False):
+        max_in_flight_calls: int = 2, device: str = "cuda:0", collect_scores: bool = False, model=None):
+    import time
     import torch
     from . import runtime as rt
 
-    shape = shape or synth.workload(5).model
+    t_setup = time.perf_counter()
+    own_model = model is None
+    if own_model:
+        shape = shape or synth.workload(5).model
+        w = synth.make_weights(shape, seed)
+        model = rt.Model(shape, w, device)
+    else:
+        shape, w = model.shape, None
     rng = np.random.default_rng(seed)
-    w = synth.make_weights(shape, seed)
-    model = rt.Model(shape, w, device)
     pages_per_user = synth.pages_for(prefix)
     pool = rt.KvPool(model, hbm_users * pages_per_user, population * pages_per_user)
     B.relaygr_kv_set_max_inflight_reloads(pool.pool, max(64, 2 * batch))
     model.reserve(batch * max(prefix, n_short + n_cand), batch, batch * pages_per_user)
     zipf = synth.ZipfIds(shape.vocab, 1.1)
     main, side = torch.cuda.current_stream(), torch.cuda.Stream()
+    clock = torch.cuda.Stream()          # carries nothing but the arrival time stamps: an event on an idle stream completes at once
 
     # ---- every user pre-inferred once, then spilled to the DRAM tier
     for u0 in range(0, population, batch):
@@ -64,6 +71,7 @@ def run(population: int = 1024, hbm_users: int = 256, prefix: int = 4096, batch:
             pool.evict(int(u), True, side)
     torch.cuda.synchronize()
     st0 = pool.stats()
+    setup_s = time.perf_counter() - t_setup
 
     # ---- the request stream
     lru: "OrderedDict[int, None]" = OrderedDict()          # resident users, least recently used first
@@ -89,7 +97,9 @@ def run(population: int = 1024, hbm_users: int = 256, prefix: int = 4096, batch:
             done[i - max_in_flight_calls].synchronize()         # bounded queue of calls in flight
         users = popularity.draw_call(rng, batch)
         in_call = set(int(u) for u in users)
-        arrive[i].record(side)
+        # the call's arrival: stamped on the idle stream, so that queueing behind the previous call's reloads counts as latency
+        arrive[i].record(clock)
+        pages_free = None
         for u in in_call:                                         # the pseudo pre-infer probe: HBM, then DRAM
             tier, _ = pool.lookup(u)
             if tier == B.TIER_HBM:
@@ -98,12 +108,16 @@ def run(population: int = 1024, hbm_users: int = 256, prefix: int = 4096, batch:
                 tiers["loading"] += 1
             elif tier == B.TIER_HOST:
                 tiers["host"] += 1
-                while pool.stats()["pages_free"] < pages_per_user:      # sliding window: make room
+                if pages_free is None:
+                    pages_free = pool.stats()["pages_free"]             # read once per call, then counted
+                while pages_free < pages_per_user:                       # sliding window: make room
                     victim = next(v for v in lru if v not in in_call)
                     pool.evict(victim, False, side)                       # its DRAM copy stays
                     del lru[victim]
+                    pages_free += pages_per_user
                 code, _ = pool.reload(u, side)
                 assert code == B.OK
+                pages_free -= pages_per_user
             else:
                 raise RuntimeError("user %d has no cache in any tier" % u)
             lru[u] = None
@@ -135,11 +149,14 @@ def run(population: int = 1024, hbm_users: int = 256, prefix: int = 4096, batch:
         "reloads": st1["reloads"] - st_w["reloads"], "reload_bytes": reload_bytes,
         "pcie_gb_per_s": reload_bytes / (wall_ms * 1e-3) / 1e9,
         "hbm_kv_gb_per_s": calls * batch * shape.kv_bytes(prefix) / (wall_ms * 1e-3) / 1e9,
-        "spilled_at_start": st0["users_host"], "ms_total": wall_ms,
+        "spilled_at_start": st0["users_host"], "ms_total": wall_ms, "setup_s": setup_s,
+        "latency_clock": "from the call's arrival (an event on an idle stream, before its probes and reloads are enqueued) to the end of its rank",
     }
     result = (report, kept, (model, pool, w, rotations)) if collect_scores else report
     if not collect_scores:
-        pool.close(); model.close()
+        pool.close()
+        if own_model:
+            model.close()
     return result
 
 

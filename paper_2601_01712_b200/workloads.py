@@ -108,15 +108,23 @@ class Built:
 
 def build(shape: synth.ModelShape, seed: int, p_lens, s_lens, c_lens, n_rotations: int = 8, zipf_a: float = 1.1,
           shuffle_pages: bool = False, spare_pages: int = 0, host_pages: int = 0, first_user: int = 0,
-          weights: Optional[synth.Weights] = None, device: str = "cuda:0") -> Built:
+          weights: Optional[synth.Weights] = None, device: str = "cuda:0", model=None, user_ids=None) -> Built:
     """Model + pool + ``n_rotations`` batches with the given per-user lengths; users are ALLOCATED
-    (not yet pre-inferred).  ``shuffle_pages`` scatters each user's pages with a seeded shuffle."""
+    (not yet pre-inferred).  ``shuffle_pages`` scatters each user's pages with a seeded shuffle.
+    ``model``: reuse an existing runtime.Model (its weights and context) instead of uploading a new one.
+    ``user_ids``: the users' ids (default: first_user, first_user + 1, ...)."""
     from . import runtime as rt
-    w = weights if weights is not None else synth.make_weights(shape, seed)
-    model = rt.Model(shape, w, device)
+    if model is not None:
+        w = weights
+    else:
+        w = weights if weights is not None else synth.make_weights(shape, seed)
+        model = rt.Model(shape, w, device)
     rng = np.random.default_rng(seed)
     zipf = synth.ZipfIds(shape.vocab, zipf_a)
     first = synth.make_batch(zipf, rng, p_lens, s_lens, c_lens, first_user)
+    if user_ids is not None:
+        assert len(user_ids) == len(p_lens) and len(set(int(u) for u in user_ids)) == len(p_lens)
+        first.users = np.asarray(user_ids, dtype=np.uint64)
     batches = [first] + [synth.draw_short_cand(zipf, rng, first) for _ in range(n_rotations - 1)]
     counts = [synth.pages_for(p) for p in p_lens]
     total = sum(counts) + spare_pages

@@ -53,11 +53,30 @@ def test_static_scratch_matches_lent_workspace_on_two_calls_in_a_row(kind):
         got = got.cpu().numpy()
         assert np.all(np.isfinite(got))
         assert float(np.max(np.abs(got - expect))) <= tol
-    # a lent workspace is left alone, and receives the (healthy) status
+    # a lent workspace is left alone (beyond its status word), and receives the (healthy) status
     model.reserve(64, 1, 0)
-    got = _scores_static(B, model, rt.DeviceBatch(batches[1], model.device))
+    model._ws[1024:].fill_(0xA7)
+    db1, db0 = rt.DeviceBatch(batches[1], model.device), rt.DeviceBatch(batches[0], model.device)
+    got = _scores_static(B, model, db1)
     assert model.device_status() == 0
     assert float(np.max(np.abs(got.cpu().numpy() - want[1]))) <= tol
+    assert bool(torch.all(model._ws[1024:] == 0xA7)), "the lent workspace was written"
+    # nothing is allocated on the device by a call (the set-up of the first call is over by now), and two calls queued
+    # back to back on one stream without a synchronisation in between share the array in order
+    torch.cuda.synchronize()
+    free0, alloc0 = torch.cuda.mem_get_info()[0], torch.cuda.memory_allocated()
+    out0 = torch.full((int(db0.cand_off[-1]),), float("nan"), dtype=torch.float32, device=model.device)
+    out1 = torch.full((int(db1.cand_off[-1]),), float("nan"), dtype=torch.float32, device=model.device)
+    free1, alloc1 = torch.cuda.mem_get_info()[0], torch.cuda.memory_allocated()
+    s = torch.cuda.current_stream().cuda_stream
+    for db, out in ((db0, out0), (db1, out1)):
+        B.relaygr_rank_full_static(model.ctx, db.n_users, db.prefix_ids.data_ptr(), db.prefix_off, db.short_ids.data_ptr(),
+                                   db.short_off, db.cand_ids.data_ptr(), db.cand_off, out.data_ptr(), s)
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] == free1 and torch.cuda.memory_allocated() == alloc1
+    assert free1 <= free0 and alloc1 >= alloc0
+    assert float(np.max(np.abs(out0.cpu().numpy() - want[0]))) <= tol
+    assert float(np.max(np.abs(out1.cpu().numpy() - want[1]))) <= tol
     model.close()
 
 
