@@ -408,9 +408,10 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             const int64_t row = (int64_t)sd.q_row0 + it.q0 + r;
             if (row_ok && is_cand && it.with_self) {
                 // the candidate's own key / value row, folded into the running softmax on CUDA cores
+                const int64_t self = (int64_t)sd.self_row0 + it.q0 + r;
                 const uint4 *qp = reinterpret_cast<const uint4 *>(q + row * d_model + it.head * kDh);
-                const uint4 *kp = reinterpret_cast<const uint4 *>(k_lin + row * d_model + it.head * kDh);
-                const uint4 *vp = reinterpret_cast<const uint4 *>(v_lin + row * d_model + it.head * kDh);
+                const uint4 *kp = reinterpret_cast<const uint4 *>(k_lin + self * d_model + it.head * kDh);
+                const uint4 *vp = reinterpret_cast<const uint4 *>(v_lin + self * d_model + it.head * kDh);
                 float dot = 0.f;
 #pragma unroll
                 for (int i = 0; i < 8; ++i) {

@@ -79,6 +79,7 @@ int Forward::init_device(int dev, std::string &err)
             const __nv_bfloat16 *wq = (const __nv_bfloat16 *)w.w_qkv + (size_t)l * 3 * d * d;
             int rc = make_tmap_2d_bf16(&wmaps[(size_t)l].qkv, wq, 3 * d, d, d, (uint32_t)kGemmWeightBoxRows, 64);
             rc |= make_tmap_2d_bf16(&wmaps[(size_t)l].kv, wq + d * d, 2 * d, d, d, (uint32_t)kGemmWeightBoxRows, 64);
+            rc |= make_tmap_2d_bf16(&wmaps[(size_t)l].wq, wq, d, d, d, (uint32_t)kGemmWeightBoxRows, 64);
             rc |= make_tmap_2d_bf16(&wmaps[(size_t)l].wo, (const __nv_bfloat16 *)w.w_o + (size_t)l * d * d, d, d, d, (uint32_t)kGemmWeightBoxRows, 64);
             rc |= make_tmap_2d_bf16(&wmaps[(size_t)l].w1, (const __nv_bfloat16 *)w.w1 + (size_t)l * F * d, F, d, d, (uint32_t)kGemmWeightBoxRows, 64);
             rc |= make_tmap_2d_bf16(&wmaps[(size_t)l].w2, (const __nv_bfloat16 *)w.w2 + (size_t)l * d * F, d, F, F, (uint32_t)kGemmWeightBoxRows, 64);
@@ -128,10 +129,13 @@ WorkspaceLayout Forward::layout(int64_t rows, int64_t users, int64_t pages) cons
     l.v = take(r * d * es);
     l.att = take(r * d * es);
     l.hid = take(r * F * es);
+    l.x_c = take(r * d * 4);          // the candidate rows of x and of LN1(x), moved together (last layer of a rank call)
+    l.a_c = take(r * d * es);
     l.partial_bytes = (size_t)kMaxSplitTiles * 128 * (size_t)(cfg.d_head + 4) * 4;      // rows of m, l, two unused, O (see attention_merge_kernel)
     l.partial = take(l.partial_bytes);
     const size_t n_items = (size_t)cfg.n_heads * ((size_t)rows / 128 + (size_t)users + 1) + 2 * (size_t)kMaxSplitTiles;
-    l.meta_bytes = 4 * (((size_t)users + 1) * 5 + (size_t)users * (sizeof(SeqDesc) / 4) + (size_t)pages + n_items * (sizeof(AttnItem) / 4) + 64);
+    // two descriptor arrays and two work lists: all rows, and the candidate rows of the last layer
+    l.meta_bytes = 4 * (((size_t)users + 1) * 5 + 2 * (size_t)users * (sizeof(SeqDesc) / 4) + (size_t)pages + 2 * n_items * (sizeof(AttnItem) / 4) + 64);
     l.meta = take(l.meta_bytes);
     l.total = at;
     return l;
@@ -195,28 +199,20 @@ int Forward::run_t(const CallDesc &call, float *scores, cudaStream_t stream, std
     if (R == 0) return RELAYGR_OK;
     const int d = cfg.d_model, F = cfg.d_ff, L = cfg.n_layers, H = cfg.n_heads;
     const WorkspaceLayout lay = layout(R, B, (int64_t)call.page_table.size());
+    constexpr bool kTensor = sizeof(T) == 2;      // bf16 model: GEMMs and attention run on the tensor cores
+    const bool preinfer = call.mode == MODE_PREINFER;
+    const int64_t n_scores = (!preinfer && call.score_off) ? call.score_off[B] : 0;
+    // The last layer of a rank / full-inference call (bf16 model): only the candidates' hidden states are read afterwards, so
+    // every other row needs nothing but its K and V there.  The candidate rows are moved together and the layer's query
+    // projection, attention, output projection and feed-forward run on those rows alone.
+    const bool compact_last = kTensor && !preinfer;
 
-    // ---- metadata blob: row_off | seg_off x3 | score_off | SeqDesc[] | page table
-    std::vector<int32_t> blob;
-    auto put = [&](const int32_t *p, size_t n) { const size_t o = blob.size(); blob.insert(blob.end(), p, p + n); return o; };
-    std::vector<int32_t> row_off((size_t)B + 1);
-    for (int i = 0; i < B; ++i) row_off[(size_t)i] = call.seqs[(size_t)i].q_row0;
-    row_off[(size_t)B] = (int32_t)R;
-    const size_t o_row = put(row_off.data(), (size_t)B + 1);
-    size_t o_seg[3] = {0, 0, 0};
-    for (int s = 0; s < 3; ++s) if (call.seg_off[s]) o_seg[s] = put(call.seg_off[s], (size_t)B + 1);
-    const size_t o_score = call.score_off ? put(call.score_off, (size_t)B + 1) : 0;
-    const size_t o_seq = put(reinterpret_cast<const int32_t *>(call.seqs.data()), (size_t)B * (sizeof(SeqDesc) / 4));
-    const size_t o_pt = call.page_table.empty() ? 0 : put(call.page_table.data(), call.page_table.size());
-    // tensor-core attention work items (bf16 model): one per (user, head, 128-row tile[, KV split])
-    std::vector<AttnItem> items;
-    std::vector<AttnMerge> merges;
-    size_t o_items = 0, o_merges = 0;
-    if (sizeof(T) == 2) {
+    // ---- tensor-core attention work items: one per (user, head, 128-row tile[, KV split]) of the rows in `seqs`
+    auto build_items = [&](const std::vector<SeqDesc> &seqs, std::vector<AttnItem> &items, std::vector<AttnMerge> &merges) {
         struct Tile { int seq, q0, n_q, nb; };
         std::vector<Tile> tiles;
-        for (int u = 0; u < B; ++u) {
-            const SeqDesc &sd = call.seqs[(size_t)u];
+        for (int u = 0; u < (int)seqs.size(); ++u) {
+            const SeqDesc &sd = seqs[(size_t)u];
             const int nPB = (sd.n_paged + 63) / 64, nLB = (sd.n_lin + 63) / 64;      // key blocks of 64 (one page each)
             for (int q0 = 0; q0 < sd.n_q; q0 += 128) {
                 const int n_q = std::min(128, sd.n_q - q0);
@@ -248,7 +244,7 @@ int Forward::run_t(const CallDesc &call, float *scores, cudaStream_t stream, std
         for (const Tile &t : tiles) {
             int ns = std::max(1, std::min(want, t.nb / 8));          // at least 8 key blocks (512 keys) per split
             if (ns > 1 && part_slot + ns * H > kMaxSplitTiles) ns = 1;
-            const bool has_cand = call.seqs[(size_t)t.seq].q_pos0 + t.q0 + t.n_q > call.seqs[(size_t)t.seq].causal_end;
+            const bool has_cand = seqs[(size_t)t.seq].q_pos0 + t.q0 + t.n_q > seqs[(size_t)t.seq].causal_end;
             for (int h = 0; h < H; ++h) {
                 if (ns == 1) {
                     items.push_back({t.seq, h, t.q0, t.n_q, 0, t.nb, -1, has_cand ? 1 : 0});
@@ -262,8 +258,43 @@ int Forward::run_t(const CallDesc &call, float *scores, cudaStream_t stream, std
                 }
             }
         }
+    };
+
+    // ---- metadata blob: row_off | seg_off x3 | score_off | SeqDesc[] | page table | attention items [| the same for the last layer]
+    std::vector<int32_t> blob;
+    auto put = [&](const int32_t *p, size_t n) { const size_t o = blob.size(); blob.insert(blob.end(), p, p + n); return o; };
+    std::vector<int32_t> row_off((size_t)B + 1);
+    for (int i = 0; i < B; ++i) row_off[(size_t)i] = call.seqs[(size_t)i].q_row0;
+    row_off[(size_t)B] = (int32_t)R;
+    const size_t o_row = put(row_off.data(), (size_t)B + 1);
+    size_t o_seg[3] = {0, 0, 0};
+    for (int s = 0; s < 3; ++s) if (call.seg_off[s]) o_seg[s] = put(call.seg_off[s], (size_t)B + 1);
+    const size_t o_score = call.score_off ? put(call.score_off, (size_t)B + 1) : 0;
+    const size_t o_seq = put(reinterpret_cast<const int32_t *>(call.seqs.data()), (size_t)B * (sizeof(SeqDesc) / 4));
+    const size_t o_pt = call.page_table.empty() ? 0 : put(call.page_table.data(), call.page_table.size());
+    std::vector<AttnItem> items, items_c;
+    std::vector<AttnMerge> merges, merges_c;
+    std::vector<SeqDesc> seqs_c;                  // the candidates of each user as rows of their own (last layer)
+    size_t o_items = 0, o_merges = 0, o_seq_c = 0, o_items_c = 0, o_merges_c = 0;
+    if (kTensor) {
+        build_items(call.seqs, items, merges);
         if (!items.empty()) o_items = put(reinterpret_cast<const int32_t *>(items.data()), items.size() * (sizeof(AttnItem) / 4));
         if (!merges.empty()) o_merges = put(reinterpret_cast<const int32_t *>(merges.data()), merges.size() * (sizeof(AttnMerge) / 4));
+        if (compact_last && n_scores > 0) {
+            seqs_c = call.seqs;
+            for (int u = 0; u < B; ++u) {
+                SeqDesc &c = seqs_c[(size_t)u];
+                c.self_row0 = c.score_row0;           // where the candidates' own K / V rows (and their x, a rows) are
+                c.q_row0 = call.score_off[u];         // where their rows are once moved together
+                c.n_q = c.n_score;
+                c.q_pos0 = c.causal_end;              // every row is a candidate
+                c.score_row0 = call.score_off[u];
+            }
+            o_seq_c = put(reinterpret_cast<const int32_t *>(seqs_c.data()), (size_t)B * (sizeof(SeqDesc) / 4));
+            build_items(seqs_c, items_c, merges_c);
+            if (!items_c.empty()) o_items_c = put(reinterpret_cast<const int32_t *>(items_c.data()), items_c.size() * (sizeof(AttnItem) / 4));
+            if (!merges_c.empty()) o_merges_c = put(reinterpret_cast<const int32_t *>(merges_c.data()), merges_c.size() * (sizeof(AttnMerge) / 4));
+        }
     }
     if (blob.size() * 4 > lay.meta_bytes) { err = "internal: metadata larger than its workspace region"; return RELAYGR_E_NOSPACE; }
     int rc = upload(blob, lay.meta, stream, err);
@@ -281,20 +312,18 @@ int Forward::run_t(const CallDesc &call, float *scores, cudaStream_t stream, std
     src.row_off = d_row_off;
     src.n_users = B;
 
-    float *x = reinterpret_cast<float *>(ws + lay.x);
-    T *a = reinterpret_cast<T *>(ws + lay.a), *q = reinterpret_cast<T *>(ws + lay.q);
+    float *x = reinterpret_cast<float *>(ws + lay.x), *x_c = reinterpret_cast<float *>(ws + lay.x_c);
+    T *a = reinterpret_cast<T *>(ws + lay.a), *q = reinterpret_cast<T *>(ws + lay.q), *a_c = reinterpret_cast<T *>(ws + lay.a_c);
     T *kl = reinterpret_cast<T *>(ws + lay.k), *vl = reinterpret_cast<T *>(ws + lay.v);
     T *att = reinterpret_cast<T *>(ws + lay.att), *hid = reinterpret_cast<T *>(ws + lay.hid);
-    const bool preinfer = call.mode == MODE_PREINFER;
 
     cudaError_t e = cudaSuccess;
     auto ck = [&](const char *what) -> bool { if (e != cudaSuccess) { err = cuda_msg(what, e); return false; } return true; };
 
-    // bf16 model: GEMMs and attention run on the tensor cores; per-call tensor maps of the activations
-    constexpr bool kTensor = sizeof(T) == 2;
+    // per-call tensor maps of the activations (bf16 model)
     int *d_status = reinterpret_cast<int *>(ws + lay.status);
-    CUtensorMap tm_a, tm_att, tm_hid, tm_q, tm_k, tm_v, tm_pool;
-    GemmOutMaps om_qkv{}, om_hid{}, om_x{};
+    CUtensorMap tm_a, tm_a_c, tm_att, tm_hid, tm_q, tm_k, tm_v, tm_pool;
+    GemmOutMaps om_qkv{}, om_hid{}, om_x{}, om_x_c{};
     if (kTensor) {
         int trc = make_tmap_2d_bf16(&tm_a, a, (uint64_t)R, (uint64_t)d, (uint64_t)d, 128, 64);
         trc |= make_tmap_2d_bf16(&tm_att, att, (uint64_t)R, (uint64_t)d, (uint64_t)d, 128, 64);
@@ -318,38 +347,56 @@ int Forward::run_t(const CallDesc &call, float *scores, cudaStream_t stream, std
             om_qkv.pool = om_qkv.o[0];
         om_hid.o[1] = om_hid.o[2] = om_hid.pool = om_hid.o[0];
         om_x.o[1] = om_x.o[2] = om_x.pool = om_x.o[0];
+        if (compact_last && n_scores > 0) {
+            trc |= make_tmap_2d_bf16(&tm_a_c, a_c, (uint64_t)n_scores, (uint64_t)d, (uint64_t)d, 128, 64);
+            trc |= make_tmap_2d_f32(&om_x_c.o[0], x_c, (uint64_t)n_scores, (uint64_t)d, (uint64_t)d, 32, 32);
+            om_x_c.o[1] = om_x_c.o[2] = om_x_c.pool = om_x_c.o[0];
+        }
         if (trc != 0) { err = "tensor-map encoding of the activations failed"; return RELAYGR_E_CUDA; }
     }
-    auto gemm = [&](const T *A, const CUtensorMap &tmA, const T *W, const CUtensorMap *tmW, const GemmOutMaps &om, int N, int K,
+    auto gemm = [&](int64_t M, const T *A, const CUtensorMap &tmA, const T *W, const CUtensorMap *tmW, const GemmOutMaps &om, int N, int K,
                     const Epilogue &ep) {
         cudaEvent_t pe = prof_begin(stream);
         cudaError_t r;
-        if constexpr (kTensor) r = launch_gemm_tc(tmA, *tmW, om, R, N, K, ep, d_status, stream, &launches);
-        else r = launch_gemm_simt<T>(A, W, R, N, K, ep, stream, &launches);
+        if constexpr (kTensor) r = launch_gemm_tc(tmA, *tmW, om, M, N, K, ep, d_status, stream, &launches);
+        else r = launch_gemm_simt<T>(A, W, M, N, K, ep, stream, &launches);
         prof_end(KC_GEMM, pe, stream);
         return r;
     };
-    auto layernorm = [&](const float *g, const float *b) {
+    auto layernorm = [&](const float *xin, int64_t M, const float *g, const float *b) {
         cudaEvent_t pe = prof_begin(stream);
-        const cudaError_t r = launch_layernorm<T>(x, d, R, g, b, cfg.ln_eps, a, stream, &launches);
+        const cudaError_t r = launch_layernorm<T>(xin, d, M, g, b, cfg.ln_eps, a, stream, &launches);
         prof_end(KC_LAYERNORM, pe, stream);
         return r;
     };
     const LayerMaps *lm = nullptr;
 
+    // the rows the part of a layer after the QKV projection runs on: all of them, or (last layer) the candidates alone
+    int64_t M = R;
+    float *xm = x;
+    const GemmOutMaps *om_xm = &om_x;
+    const SeqDesc *seqs_m = d_seqs;
+    const AttnItem *items_m = reinterpret_cast<const AttnItem *>(meta + o_items);
+    const AttnMerge *merges_m = reinterpret_cast<const AttnMerge *>(meta + o_merges);
+    int n_items_m = (int)items.size(), n_merges_m = (int)merges.size();
+    bool dead_tail = false;                       // a call without candidates: nothing reads the last layer
+
     for (int l = 0; l < L; ++l) {
+        const bool last = l == L - 1;
+        if (last && !preinfer && n_scores == 0) { dead_tail = true; break; }
         const float *g1 = w.ln1_g + (size_t)l * d, *b1n = w.ln1_b + (size_t)l * d;
         if (l == 0) {
             cudaEvent_t pe = prof_begin(stream);
-            e = launch_gather_ln<T>((const T *)w.emb, cfg.vocab, d, src, R, g1, b1n, cfg.ln_eps, x, a, reinterpret_cast<int *>(ws + lay.status), stream, &launches);
+            e = launch_gather_ln<T>((const T *)w.emb, cfg.vocab, d, src, R, g1, b1n, cfg.ln_eps, x, a, d_status, stream, &launches);
             prof_end(KC_GATHER_LN, pe, stream);
         } else {
-            e = layernorm(g1, b1n);
+            e = layernorm(x, R, g1, b1n);
         }
         if (!ck("LayerNorm 1")) return RELAYGR_E_CUDA;
 
-        // fused QKV projection; the last pre-infer layer only needs K and V (psi is K/V alone)
-        const bool kv_only = preinfer && l == L - 1;
+        // fused QKV projection over all rows; K and V only in the last pre-infer layer (psi is K/V alone) and in the last
+        // layer of a rank call (the queries of the candidates follow below, on their rows alone)
+        const bool kv_only = last && (preinfer || compact_last);
         Epilogue ep{};
         ep.mode = EPI_QKV;
         ep.col0 = kv_only ? d : 0;
@@ -364,16 +411,37 @@ int Forward::run_t(const CallDesc &call, float *scores, cudaStream_t stream, std
         if (preinfer) ep.paged = paged;
         const T *Wqkv = (const T *)w.w_qkv + ((size_t)l * 3 * d + ep.col0) * d;
         lm = kTensor ? &wmaps[(size_t)l] : nullptr;
-        e = gemm(a, tm_a, Wqkv, lm ? (kv_only ? &lm->kv : &lm->qkv) : nullptr, om_qkv, 3 * d - ep.col0, d, ep);
+        e = gemm(R, a, tm_a, Wqkv, lm ? (kv_only ? &lm->kv : &lm->qkv) : nullptr, om_qkv, 3 * d - ep.col0, d, ep);
         if (!ck("QKV projection")) return RELAYGR_E_CUDA;
-        if (kv_only) break;
+        if (preinfer && last) break;
+
+        if (last && compact_last) {
+            // move the candidates' rows of x and of LN1(x) together, then project their queries
+            M = n_scores; xm = x_c; om_xm = &om_x_c;
+            seqs_m = reinterpret_cast<const SeqDesc *>(meta + o_seq_c);
+            items_m = reinterpret_cast<const AttnItem *>(meta + o_items_c);
+            merges_m = reinterpret_cast<const AttnMerge *>(meta + o_merges_c);
+            n_items_m = (int)items_c.size(); n_merges_m = (int)merges_c.size();
+            cudaEvent_t pe = prof_begin(stream);
+            e = launch_compact_rows<T>(x, a, seqs_m, B, meta + o_score, n_scores, d, x_c, a_c, stream, &launches);
+            prof_end(KC_LAYERNORM, pe, stream);
+            if (!ck("candidate rows")) return RELAYGR_E_CUDA;
+            Epilogue eq{};
+            eq.mode = EPI_QKV;
+            eq.col0 = 0;
+            eq.bias = w.b_qkv ? w.b_qkv + (size_t)l * 3 * d : nullptr;
+            eq.d_model = d;
+            eq.q = q; eq.k_lin = kl; eq.v_lin = vl;
+            eq.seqs = seqs_m; eq.row_off = meta + o_score; eq.n_users = B;
+            e = gemm(M, a_c, tm_a_c, (const T *)w.w_qkv + (size_t)l * 3 * d * d, lm ? &lm->wq : nullptr, om_qkv, d, d, eq);
+            if (!ck("query projection")) return RELAYGR_E_CUDA;
+        }
 
         {
             cudaEvent_t pe = prof_begin(stream);
             if constexpr (kTensor)
-                e = launch_attention_tc(tm_q, tm_k, tm_v, tm_pool, reinterpret_cast<const AttnItem *>(meta + o_items), (int)items.size(),
-                                        reinterpret_cast<const AttnMerge *>(meta + o_merges), (int)merges.size(), d_seqs, meta + o_pt, L,
-                                        l, d, q, kl, vl, cfg.attn_kind, (!preinfer && l == L - 1) ? 1 : 0, att, reinterpret_cast<float *>(ws + lay.partial), d_status,
+                e = launch_attention_tc(tm_q, tm_k, tm_v, tm_pool, items_m, n_items_m, merges_m, n_merges_m, seqs_m, meta + o_pt, L,
+                                        l, d, q, kl, vl, cfg.attn_kind, 0, att, reinterpret_cast<float *>(ws + lay.partial), d_status,
                                         stream, &launches);
             else
                 e = launch_attention_simt<T>(q, kl, vl, paged, d_seqs, d_row_off, B, R, H, cfg.d_head, cfg.attn_kind, att, stream, &launches);
@@ -384,35 +452,35 @@ int Forward::run_t(const CallDesc &call, float *scores, cudaStream_t stream, std
         if (kTensor && ffn_fused_supported((int)d, (int)F)) {
             // output projection + residual, LayerNorm 2, both feed-forward GEMMs, SiLU and the second residual add in one kernel
             cudaEvent_t pe = prof_begin(stream);
-            e = launch_ffn_fused(lm->w1, lm->w2_wide, om_x.o[0], x, w.ln2_g + (size_t)l * d, w.ln2_b + (size_t)l * d,
+            e = launch_ffn_fused(lm->w1, lm->w2_wide, om_xm->o[0], xm, w.ln2_g + (size_t)l * d, w.ln2_b + (size_t)l * d,
                                  w.b1 ? w.b1 + (size_t)l * F : nullptr, w.b2 ? w.b2 + (size_t)l * d : nullptr, &tm_att, &lm->wo_wide,
-                                 w.b_o ? w.b_o + (size_t)l * d : nullptr, R, (int)F, cfg.ln_eps, d_status, stream, &launches);
+                                 w.b_o ? w.b_o + (size_t)l * d : nullptr, M, (int)F, cfg.ln_eps, d_status, stream, &launches);
             prof_end(KC_GEMM, pe, stream);
             if (!ck("output projection + feed-forward")) return RELAYGR_E_CUDA;
             continue;
         }
         Epilogue eo{};
-        eo.mode = EPI_RESID; eo.bias = w.b_o ? w.b_o + (size_t)l * d : nullptr; eo.resid = x; eo.out_f32 = x;
-        e = gemm(att, tm_att, (const T *)w.w_o + (size_t)l * d * d, lm ? &lm->wo : nullptr, om_x, d, d, eo);
+        eo.mode = EPI_RESID; eo.bias = w.b_o ? w.b_o + (size_t)l * d : nullptr; eo.resid = xm; eo.out_f32 = xm;
+        e = gemm(M, att, tm_att, (const T *)w.w_o + (size_t)l * d * d, lm ? &lm->wo : nullptr, *om_xm, d, d, eo);
         if (!ck("output projection")) return RELAYGR_E_CUDA;
 
-        e = layernorm(w.ln2_g + (size_t)l * d, w.ln2_b + (size_t)l * d);
+        e = layernorm(xm, M, w.ln2_g + (size_t)l * d, w.ln2_b + (size_t)l * d);
         if (!ck("LayerNorm 2")) return RELAYGR_E_CUDA;
 
         Epilogue e1{};
         e1.mode = EPI_STORE; e1.silu = 1; e1.bias = w.b1 ? w.b1 + (size_t)l * F : nullptr; e1.out = hid;
-        e = gemm(a, tm_a, (const T *)w.w1 + (size_t)l * F * d, lm ? &lm->w1 : nullptr, om_hid, F, d, e1);
+        e = gemm(M, a, tm_a, (const T *)w.w1 + (size_t)l * F * d, lm ? &lm->w1 : nullptr, om_hid, F, d, e1);
         if (!ck("FFN 1")) return RELAYGR_E_CUDA;
 
         Epilogue e2{};
-        e2.mode = EPI_RESID; e2.bias = w.b2 ? w.b2 + (size_t)l * d : nullptr; e2.resid = x; e2.out_f32 = x;
-        e = gemm(hid, tm_hid, (const T *)w.w2 + (size_t)l * d * F, lm ? &lm->w2 : nullptr, om_x, d, F, e2);
+        e2.mode = EPI_RESID; e2.bias = w.b2 ? w.b2 + (size_t)l * d : nullptr; e2.resid = xm; e2.out_f32 = xm;
+        e = gemm(M, hid, tm_hid, (const T *)w.w2 + (size_t)l * d * F, lm ? &lm->w2 : nullptr, *om_xm, d, F, e2);
         if (!ck("FFN 2")) return RELAYGR_E_CUDA;
     }
 
-    if (!preinfer && call.score_off && call.score_off[B] > 0) {
+    if (!dead_tail && n_scores > 0) {
         cudaEvent_t pe = prof_begin(stream);
-        e = launch_score(x, d, d_seqs, B, call.score_off[B], meta + o_score, w.lnf_g, w.lnf_b, cfg.ln_eps, w.w_score, w.b_score,
+        e = launch_score(xm, d, seqs_m, B, n_scores, meta + o_score, w.lnf_g, w.lnf_b, cfg.ln_eps, w.w_score, w.b_score,
                          scores, stream, &launches);
         prof_end(KC_SCORE, pe, stream);
         if (!ck("scoring head")) return RELAYGR_E_CUDA;

@@ -29,7 +29,7 @@ struct CallDesc {
 };
 
 struct WorkspaceLayout {
-    size_t status, x, a, q, k, v, att, hid, partial, meta, total;
+    size_t status, x, a, q, k, v, att, hid, x_c, a_c, partial, meta, total;
     size_t meta_bytes, partial_bytes;
 };
 
@@ -43,7 +43,7 @@ struct Forward {
     int n_sms = 148;
 
     // tensor maps of the weights (bf16 model), one set per layer
-    struct LayerMaps { CUtensorMap qkv, kv, wo, w1, w2, w2_wide, wo_wide; };      // *_wide: boxes of 256 rows (fused out-proj + feed-forward)
+    struct LayerMaps { CUtensorMap qkv, kv, wq, wo, w1, w2, w2_wide, wo_wide; };      // *_wide: boxes of 256 rows (fused out-proj + feed-forward)
     std::vector<LayerMaps> wmaps;
 
     // pinned staging ring for the per-call metadata

@@ -15,13 +15,16 @@ namespace relaygr {
 // "linear" keys (rows of the call's transient K/V buffers) at positions
 // lin_pos0 .. lin_pos0+n_lin-1.  Mask: a query at position t < causal_end sees
 // keys at positions <= t; a query at t >= causal_end (a candidate) sees keys at
-// positions < causal_end plus its own K/V row.
+// positions < causal_end plus its own K/V row, which is row self_row0 + i of the transient K/V buffers for the user's
+// query row i (the query rows themselves may sit elsewhere: the last layer of a rank call runs on the candidate rows alone,
+// moved together, while their K/V stay where the projection of all rows wrote them).
 struct SeqDesc {
     int32_t q_row0, n_q, q_pos0;
     int32_t n_paged, pt_base;
     int32_t lin_row0, n_lin, lin_pos0;
     int32_t causal_end;
     int32_t score_row0, n_score, score_out0;
+    int32_t self_row0;
 };
 
 // Where the token ids of the rows come from: up to three jagged segments per user, in order.

@@ -61,6 +61,12 @@ template <typename T>
 cudaError_t launch_layernorm(const float *x, int d, int64_t n_rows, const float *g, const float *b, float eps, T *a,
                              cudaStream_t stream, int64_t *launches);
 
+// x_c[i, :] = x[row(i), :], a_c[i, :] = a[row(i), :] for the n_total candidate rows of the call in score order, where
+// row(i) = seqs[u].self_row0 + (i - score_off[u]) for the user u that candidate i belongs to (seqs: the compact descriptors).
+template <typename T>
+cudaError_t launch_compact_rows(const float *x, const T *a, const SeqDesc *seqs, int n_users, const int32_t *score_off, int64_t n_total,
+                                int d, float *x_c, T *a_c, cudaStream_t stream, int64_t *launches);
+
 // scores[score_out0 + i] = LN(x[score_row0 + i]; g, b) . w + bias for every user's candidate rows.
 cudaError_t launch_score(const float *x, int d, const SeqDesc *seqs, int n_users, int64_t n_scores_total,
                          const int32_t *score_off, const float *g, const float *b, float eps,

@@ -154,6 +154,28 @@ gather_ln_kernel(const T *__restrict__ emb, int64_t vocab, int d, RowSource src,
     ln_rows_store<T, NC, ROWS>(v, d, lane, row0, n_rows, g, b, eps, a);
 }
 
+// The candidate rows of every user, moved together: row i of x_c / a_c is the i-th candidate of the call (score order).
+// seqs holds the COMPACT descriptors: self_row0 = row of the user's first candidate in the full-row buffers.
+template <typename T>
+__global__ void __launch_bounds__(kWarpsPerBlock * 32)
+compact_rows_kernel(const float *__restrict__ x, const T *__restrict__ a, const SeqDesc *__restrict__ seqs, int n_users,
+                    const int32_t *__restrict__ score_off, int64_t n_total, int d, float *__restrict__ x_c, T *__restrict__ a_c)
+{
+    grid_launch_dependents();
+    grid_dependency_wait();
+    const int64_t i = (int64_t)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (i >= n_total) return;
+    const int u = find_user(score_off, n_users, (int)i);
+    const int64_t src = (int64_t)seqs[u].self_row0 + (i - score_off[u]);
+    const uint4 *xs = reinterpret_cast<const uint4 *>(x + src * d);
+    uint4 *xd = reinterpret_cast<uint4 *>(x_c + i * d);
+    for (int j = lane; j < d / 4; j += 32) xd[j] = xs[j];
+    const uint4 *as = reinterpret_cast<const uint4 *>(a + src * d);
+    uint4 *ad = reinterpret_cast<uint4 *>(a_c + i * d);
+    for (int j = lane; j < d * (int)sizeof(T) / 16; j += 32) ad[j] = as[j];
+}
+
 // a[r, :] = LN(x[r, :]).  A warp takes ROWS consecutive rows at once and issues all their loads before any
 // arithmetic, so that enough bytes are in flight per SM to reach HBM / L2 bandwidth; NC = chunks of 128 columns.
 template <typename T, int NC, int ROWS>
@@ -458,6 +480,16 @@ cudaError_t launch_score(const float *x, int d, const SeqDesc *seqs, int n_users
 }
 
 template <typename T>
+cudaError_t launch_compact_rows(const float *x, const T *a, const SeqDesc *seqs, int n_users, const int32_t *score_off, int64_t n_total,
+                                int d, float *x_c, T *a_c, cudaStream_t stream, int64_t *launches)
+{
+    if (n_total == 0) return cudaSuccess;
+    *launches += 1;
+    return launch_dependent(compact_rows_kernel<T>, dim3(blocks_for(n_total)), dim3(kWarpsPerBlock * 32), 0, stream, 1, x, a, seqs, n_users,
+                            score_off, n_total, d, x_c, a_c);
+}
+
+template <typename T>
 cudaError_t launch_gemm_simt(const T *A, const T *W, int64_t M, int N, int K, const Epilogue &epi, cudaStream_t stream,
                              int64_t *launches)
 {
@@ -493,6 +525,8 @@ cudaError_t launch_attention_simt(const T *q, const T *k_lin, const T *v_lin, Pa
                                              float *, T *, int *, cudaStream_t, int64_t *);                                 \
     template cudaError_t launch_layernorm<T>(const float *, int, int64_t, const float *, const float *, float, T *,          \
                                              cudaStream_t, int64_t *);                                                      \
+    template cudaError_t launch_compact_rows<T>(const float *, const T *, const SeqDesc *, int, const int32_t *, int64_t, int, \
+                                                float *, T *, cudaStream_t, int64_t *);                                     \
     template cudaError_t launch_gemm_simt<T>(const T *, const T *, int64_t, int, int, const Epilogue &, cudaStream_t,        \
                                              int64_t *);                                                                    \
     template cudaError_t launch_attention_simt<T>(const T *, const T *, const T *, PagedKV, const SeqDesc *, const int32_t *, \

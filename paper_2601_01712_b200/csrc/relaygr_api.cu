@@ -370,6 +370,7 @@ int32_t relaygr_preinfer(relaygr_ctx *ctx, relaygr_kv_pool *pool, int32_t n_user
         s.lin_row0 = 0; s.n_lin = 0; s.lin_pos0 = P;
         s.causal_end = P;
         s.score_row0 = 0; s.n_score = 0; s.score_out0 = 0;
+        s.self_row0 = s.q_row0;
         call.page_table.insert(call.page_table.end(), entries[i]->pages.begin(), entries[i]->pages.end());
         call.seqs.push_back(s);
     }
@@ -430,6 +431,7 @@ int32_t relaygr_rank(relaygr_ctx *ctx, relaygr_kv_pool *pool, int32_t n_users, c
         s.lin_row0 = row; s.n_lin = S; s.lin_pos0 = P;
         s.causal_end = P + S;
         s.score_row0 = row + S; s.n_score = C; s.score_out0 = cand_off[i];
+        s.self_row0 = s.q_row0;
         call.page_table.insert(call.page_table.end(), entries[(size_t)i]->pages.begin(), entries[(size_t)i]->pages.end());
         call.seqs.push_back(s);
         row += S + C;
@@ -481,6 +483,7 @@ int32_t relaygr_rank_full(relaygr_ctx *ctx, int32_t n_users, const int32_t *pref
         s.lin_row0 = (int32_t)row; s.n_lin = P + S; s.lin_pos0 = 0;
         s.causal_end = P + S;
         s.score_row0 = (int32_t)row + P + S; s.n_score = C; s.score_out0 = cand_off[i];
+        s.self_row0 = s.q_row0;
         call.seqs.push_back(s);
         row += P + S + C;
     }

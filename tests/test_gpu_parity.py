@@ -1,12 +1,14 @@
 """GPU parity: the CUDA path, called through the C ABI, against the CPU checker on the
 same seeded inputs.  Integer / byte work (gather, page indexing, tier copies) must be
 bit-exact; scores within 1e-4 (fp32 model) or 2e-2 (bf16 model) max-abs."""
+import os
+
 import numpy as np
 import pytest
 import torch
 
 from paper_2601_01712_b200 import synth
-from tests.helpers import TOL_BF16, TOL_BF16_POINTWISE, TOL_F32, max_abs_err, oracle_model, oracle_scores, small_bf16_shape
+from tests.helpers import TOL_BF16, TOL_F32, bf16_noise_bounds, max_abs_err, oracle_model, oracle_scores, small_bf16_shape
 
 pytestmark = pytest.mark.gpu
 
@@ -286,6 +288,22 @@ def test_config4_long_model_sampled_user():
     _full_size(4, [4096] * 16, [128] * 16, [1024] * 16, sample=[5], shuffle=False)
 
 
+@pytest.mark.parametrize("prefix,user", [(8192, 11), (16384, 3)])
+def test_config4_long_prefixes_sampled_user(prefix, user):
+    """The long-sequence workload at long prefixes, in the launch configuration the benchmark times (16 users, 8 layers,
+    d_model 512): every one of the sampled user's 1024 candidates against the checker.  Longer prefixes are not more of the
+    same for the kernels - 130 / 258 key blocks per work item, many more decisions of the stale-maximum softmax, more waves.
+    The fp64 checker's pre-infer grows with the square of the prefix: half a minute at 8192 tokens, about two minutes at
+    16384 and five at 24576 on 16 host cores, which is why the longest length here is 16384 (the 24576-token case has been
+    run with this same function and passes; set RELAYGR_TEST_P24576=1 to include it)."""
+    _full_size(4, [prefix] * 16, [128] * 16, [1024] * 16, sample=[user], shuffle=False)
+
+
+@pytest.mark.skipif(not os.environ.get("RELAYGR_TEST_P24576"), reason="five minutes of CPU checker; opt in with RELAYGR_TEST_P24576=1")
+def test_config4_longest_prefix_sampled_user():
+    _full_size(4, [24576] * 16, [128] * 16, [1024] * 16, sample=[3], shuffle=False)
+
+
 def test_reload_tier_workload_small():
     """The reload-tier workload at a reduced population: every call's scores equal those of the same users ranked
     from prefixes that never left HBM (bit for bit: spill and reload move bytes), and the tiers are accounted for."""
@@ -440,8 +458,12 @@ def test_pointwise_attention_bf16_matches_checker(case):
         assert np.max(np.abs(gK.float().cpu().numpy() - K)) <= 5e-2
         assert np.max(np.abs(gV.float().cpu().numpy() - V)) <= 5e-2
     want = oracle_scores(om, batch)
-    assert max_abs_err(scores.cpu().numpy(), batch, want) <= TOL_BF16_POINTWISE
-    assert max_abs_err(full.cpu().numpy(), batch, want) <= TOL_BF16_POINTWISE
+    # the variant's scores spread twice as wide as the softmax model's on the same weights and bf16 rounding is relative: the
+    # bound follows from the rounding noise this very model and batch must show (helpers.bf16_noise_bounds), not from a run
+    max_bound, _, sigma = bf16_noise_bounds(shape, w, batch, want)
+    assert max_bound <= 2.5 * TOL_BF16, sigma
+    assert max_abs_err(scores.cpu().numpy(), batch, want) <= max_bound
+    assert max_abs_err(full.cpu().numpy(), batch, want) <= max_bound
     assert np.std(np.concatenate([v for v in want.values() if len(v)])) > 0.3          # scores are not degenerate
     assert model.device_status() == 0
     pool.close(); model.close()
@@ -493,6 +515,11 @@ def test_sharp_logits_take_the_rescaling_path(q_gain):
     if q_gain <= 8.0:
         assert max_abs_err(scores, batch, want) <= q_gain * TOL_BF16
         assert max_abs_err(full, batch, want) <= q_gain * TOL_BF16
+        # the emulation of the unavoidable roundings on these very weights confirms the size of that error (rms about gain x
+        # the usual 0.003; its tail is heavier than a normal one here, so it is not used as the bound on the maximum)
+        _, rms_bound, sigma = bf16_noise_bounds(shape, w, batch, want)
+        err = np.concatenate([scores[batch.cand_off[i]:batch.cand_off[i + 1]] - wv for i, wv in want.items()])
+        assert np.sqrt(np.mean(err ** 2)) <= rms_bound, sigma
     else:
         assert np.all(np.isfinite(scores)) and np.all(np.isfinite(full))
         err = np.concatenate([np.abs(scores[batch.cand_off[i]:batch.cand_off[i + 1]] - wv) for i, wv in want.items()])
@@ -525,9 +552,10 @@ def _random_case(rng):
 def test_randomized_shapes_match_checker(block):
     """Seeded random models (width, depth, feed-forward width, attention variant) and jagged batches whose lengths cluster
     around the boundaries of the 64-token pages, the 128-row query tiles and the 32-row warps, half of them on shuffled
-    pages.  The error against the checker behaves like noise of rms 0.004-0.005 on scores of unit scale (bf16 rounding of
-    the activations), whose tail over a few hundred candidates reaches 4-4.5 rms: the bound on the maximum is 1.5 x the bf16
-    tolerance of the named workloads, with the rms bounded as well, so that a systematic error does not hide under it."""
+    pages.  The named workloads' bound (2e-2) is not a bound for every shape: the rounding a bf16 model cannot avoid gives
+    single-layer and narrow models score errors of rms up to 0.0065, whose largest of several hundred reaches 0.02 in a pure
+    numpy emulation with no kernel in it.  Each case is therefore held to the bounds derived from that emulation for its own
+    model and batch (helpers.bf16_noise_bounds): maximum <= max(2e-2, 5 sigma), rms <= 1.5 sigma."""
     rng = np.random.default_rng(9100 + block)
     for it in range(6):
         d, layers, ff, kind, p, s, c = _random_case(rng)
@@ -543,11 +571,12 @@ def test_randomized_shapes_match_checker(block):
         torch.cuda.synchronize()
         assert model.device_status() == 0
         want = oracle_scores(om, batch)
-        tol = TOL_BF16_POINTWISE if kind else TOL_BF16
-        case = (d, layers, ff, kind, p, s, c)
+        max_bound, rms_bound, sigma = bf16_noise_bounds(shape, w, batch, want)
+        case = (d, layers, ff, kind, p, s, c, sigma)
+        assert max_bound <= 2.5 * TOL_BF16, case                 # the yardstick itself stays in a sane range
         for got in (scores, full):
-            assert max_abs_err(got, batch, want) <= 1.5 * tol, case
+            assert max_abs_err(got, batch, want) <= max_bound, case
             err = np.concatenate([got[batch.cand_off[i]:batch.cand_off[i + 1]] - wv for i, wv in want.items()])
             if len(err):
-                assert np.sqrt(np.mean(err ** 2)) <= 0.4 * tol, case
+                assert np.sqrt(np.mean(err ** 2)) <= rms_bound, case
         pool.close(); model.close()

@@ -303,6 +303,32 @@ def test_pins_catch_planted_mistakes(mistake):
     assert np.max(np.abs(got - wrong)) > 1e-4
 
 
+# ---------------------------------------------------------------- the bf16 noise yardstick of the GPU tests
+def test_noise_emulation_without_rounding_is_the_model_and_rounding_adds_small_noise():
+    from tests import bf16_noise
+    shape = synth.ModelShape(2, 128, 2, 64, 256, 300, synth.DTYPE_BF16)
+    w = synth.make_weights(shape, 15)
+    params = {**w.mat, **w.vec}
+    m = ref.Model(shape.n_layers, shape.d_model, shape.n_heads, shape.d_head, shape.d_ff, shape.ln_eps, params)
+    rng = np.random.default_rng(27)
+    p, s, c = ids(rng, 70, 300), ids(rng, 9, 300), ids(rng, 40, 300)
+    sd = dict(shape_dict(shape), attn_kind=0)
+    want = m.full(p, s, c)
+    assert np.max(np.abs(bf16_noise.scores(sd, params, p, s, c, sites=()) - want)) <= 1e-9
+    noisy = bf16_noise.scores(sd, params, p, s, c)
+    rms = float(np.sqrt(np.mean((noisy - want) ** 2)))
+    assert 5e-4 < rms < 1e-2                                    # every site rounded: small, not zero
+    for site in bf16_noise.SITES:                               # each site alone moves the scores, by less than all together would at worst
+        e = bf16_noise.scores(sd, params, p, s, c, sites=(site,)) - want
+        assert 0 < float(np.max(np.abs(e))) < 2e-2
+    x = np.array([1.0, 1.00390625, 1.01171875, -2.5, 3.1415927, 1e-30, -65504.0])
+    assert np.array_equal(bf16_noise.bf16(x).astype(np.float32), torch.tensor(x, dtype=torch.float32).to(torch.bfloat16).float().numpy())
+    # the pointwise variant
+    m1 = ref.Model(shape.n_layers, shape.d_model, shape.n_heads, shape.d_head, shape.d_ff, shape.ln_eps, params, attn_kind=1)
+    sd1 = dict(shape_dict(shape), attn_kind=1)
+    assert np.max(np.abs(bf16_noise.scores(sd1, params, p, s, c, sites=()) - m1.full(p, s, c))) <= 1e-9
+
+
 # ---------------------------------------------------------------- input recipe
 def test_zipf_ids_are_seeded_in_range_and_skewed():
     z = synth.ZipfIds(10_000, 1.1)
