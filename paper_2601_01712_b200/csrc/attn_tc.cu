@@ -115,14 +115,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     const __grid_constant__ CUtensorMap tmVlin, const __grid_constant__ CUtensorMap tmPool,
                     const AttnItem *__restrict__ items, const SeqDesc *__restrict__ seqs, const int32_t *__restrict__ pt,
                     int n_layers, int layer, int d_model, const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restrict__ k_lin,
-                    const __nv_bfloat16 *__restrict__ v_lin, __nv_bfloat16 *__restrict__ out, float *__restrict__ partial, int only_cand, int *err)
+                    const __nv_bfloat16 *__restrict__ v_lin, __nv_bfloat16 *__restrict__ out, float *__restrict__ partial, int *err)
 {
-    if (only_cand) {
-        // last layer of a rank call: only candidate rows are read afterwards (by the scoring head), so a tile without any is skipped
-        const AttnItem it0 = items[blockIdx.x];
-        const SeqDesc s0 = seqs[it0.seq];
-        if (s0.q_pos0 + it0.q0 + it0.n_q <= s0.causal_end) return;
-    }
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t *sQ = smem;
@@ -487,12 +481,11 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
 // coalesced row segment and all rows are in flight at once (the kernel is a chain of two memory round trips).
 __global__ void __launch_bounds__(256)
 attention_merge_kernel(const AttnMerge *__restrict__ merges, const SeqDesc *__restrict__ seqs, const float *__restrict__ partial,
-                       int d_model, int only_cand, __nv_bfloat16 *__restrict__ out)
+                       int d_model, __nv_bfloat16 *__restrict__ out)
 {
     grid_launch_dependents();
     grid_dependency_wait();
     const AttnMerge mg = merges[blockIdx.x];
-    if (only_cand && seqs[mg.seq].q_pos0 + mg.q0 + mg.n_q <= seqs[mg.seq].causal_end) return;      // (see attention_tc_kernel)
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const float c = 0.125f * 1.4426950408889634f;
     const int64_t row0 = (int64_t)seqs[mg.seq].q_row0 + mg.q0;
@@ -520,7 +513,7 @@ attention_merge_kernel(const AttnMerge *__restrict__ merges, const SeqDesc *__re
 cudaError_t launch_attention_tc(const CUtensorMap &tmQ, const CUtensorMap &tmK, const CUtensorMap &tmV, const CUtensorMap &tmPool,
                                 const AttnItem *items, int n_items, const AttnMerge *merges, int n_merges, const SeqDesc *seqs,
                                 const int32_t *pt, int n_layers, int layer, int d_model, const __nv_bfloat16 *q,
-                                const __nv_bfloat16 *k_lin, const __nv_bfloat16 *v_lin, int attn_kind, int only_cand, __nv_bfloat16 *out,
+                                const __nv_bfloat16 *k_lin, const __nv_bfloat16 *v_lin, int attn_kind, __nv_bfloat16 *out,
                                 float *partial, int *err, cudaStream_t stream, int64_t *launches)
 {
     if (n_items == 0) return cudaSuccess;
@@ -537,10 +530,10 @@ cudaError_t launch_attention_tc(const CUtensorMap &tmQ, const CUtensorMap &tmK, 
     *launches += 1;
     auto kernel = attn_kind == ATTN_POINTWISE ? attention_tc_kernel<true> : attention_tc_kernel<false>;
     cudaError_t e = launch_dependent(kernel, dim3(n_items), dim3(192), (size_t)kSmemBytes, stream, 1, tmQ, tmK, tmV, tmPool, items,
-                                     seqs, pt, n_layers, layer, d_model, q, k_lin, v_lin, out, partial, only_cand, err);
+                                     seqs, pt, n_layers, layer, d_model, q, k_lin, v_lin, out, partial, err);
     if (e != cudaSuccess || n_merges == 0) return e;
     *launches += 1;
-    return launch_dependent(attention_merge_kernel, dim3(n_merges, kQTile / 8), dim3(256), 0, stream, 1, merges, seqs, partial, d_model, only_cand, out);
+    return launch_dependent(attention_merge_kernel, dim3(n_merges, kQTile / 8), dim3(256), 0, stream, 1, merges, seqs, partial, d_model, out);
 }
 
 }  // namespace relaygr

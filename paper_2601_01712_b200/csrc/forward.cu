@@ -322,9 +322,13 @@ int Forward::run_t(const CallDesc &call, float *scores, cudaStream_t stream, std
 
     // per-call tensor maps of the activations (bf16 model)
     int *d_status = reinterpret_cast<int *>(ws + lay.status);
-    CUtensorMap tm_a, tm_a_c, tm_att, tm_hid, tm_q, tm_k, tm_v, tm_pool;
-    GemmOutMaps om_qkv{}, om_hid{}, om_x{}, om_x_c{};
-    if (kTensor) {
+    CUtensorMap &tm_a = act.tm_a, &tm_a_c = act.tm_a_c, &tm_att = act.tm_att, &tm_hid = act.tm_hid, &tm_q = act.tm_q, &tm_k = act.tm_k,
+                &tm_v = act.tm_v, &tm_pool = act.tm_pool;
+    GemmOutMaps &om_qkv = act.om_qkv, &om_hid = act.om_hid, &om_x = act.om_x, &om_x_c = act.om_x_c;
+    const int64_t cand_rows = compact_last ? n_scores : 0;
+    const bool maps_cached = act.ws == ws && act.rows == R && act.cand_rows == cand_rows && act.slab == call.pool_slab && act.pages == call.pool_pages;
+    if (kTensor && !maps_cached) {
+        act.ws = nullptr;                         // not valid until every map below is encoded
         int trc = make_tmap_2d_bf16(&tm_a, a, (uint64_t)R, (uint64_t)d, (uint64_t)d, 128, 64);
         trc |= make_tmap_2d_bf16(&tm_att, att, (uint64_t)R, (uint64_t)d, (uint64_t)d, 128, 64);
         trc |= make_tmap_2d_bf16(&tm_hid, hid, (uint64_t)R, (uint64_t)F, (uint64_t)F, 128, 64);
@@ -353,6 +357,7 @@ int Forward::run_t(const CallDesc &call, float *scores, cudaStream_t stream, std
             om_x_c.o[1] = om_x_c.o[2] = om_x_c.pool = om_x_c.o[0];
         }
         if (trc != 0) { err = "tensor-map encoding of the activations failed"; return RELAYGR_E_CUDA; }
+        act.ws = ws; act.rows = R; act.cand_rows = cand_rows; act.slab = call.pool_slab; act.pages = call.pool_pages;
     }
     auto gemm = [&](int64_t M, const T *A, const CUtensorMap &tmA, const T *W, const CUtensorMap *tmW, const GemmOutMaps &om, int N, int K,
                     const Epilogue &ep) {
@@ -441,7 +446,7 @@ int Forward::run_t(const CallDesc &call, float *scores, cudaStream_t stream, std
             cudaEvent_t pe = prof_begin(stream);
             if constexpr (kTensor)
                 e = launch_attention_tc(tm_q, tm_k, tm_v, tm_pool, items_m, n_items_m, merges_m, n_merges_m, seqs_m, meta + o_pt, L,
-                                        l, d, q, kl, vl, cfg.attn_kind, 0, att, reinterpret_cast<float *>(ws + lay.partial), d_status,
+                                        l, d, q, kl, vl, cfg.attn_kind, att, reinterpret_cast<float *>(ws + lay.partial), d_status,
                                         stream, &launches);
             else
                 e = launch_attention_simt<T>(q, kl, vl, paged, d_seqs, d_row_off, B, R, H, cfg.d_head, cfg.attn_kind, att, stream, &launches);

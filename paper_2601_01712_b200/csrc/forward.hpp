@@ -11,6 +11,7 @@
 
 #include "../../include/relaygr.h"
 #include "internal.cuh"
+#include "kernels.cuh"
 
 namespace relaygr {
 
@@ -45,6 +46,14 @@ struct Forward {
     // tensor maps of the weights (bf16 model), one set per layer
     struct LayerMaps { CUtensorMap qkv, kv, wq, wo, w1, w2, w2_wide, wo_wide; };      // *_wide: boxes of 256 rows (fused out-proj + feed-forward)
     std::vector<LayerMaps> wmaps;
+
+    // tensor maps of the activations (bf16 model): a function of the workspace, the row counts and the pool slab alone, so
+    // calls of the same shape - the usual case in serving - reuse them instead of encoding some twenty maps per call
+    struct ActMaps {
+        const char *ws = nullptr; int64_t rows = -1, cand_rows = -1; const void *slab = nullptr; int64_t pages = -1;
+        CUtensorMap tm_a, tm_a_c, tm_att, tm_hid, tm_q, tm_k, tm_v, tm_pool;
+        GemmOutMaps om_qkv, om_hid, om_x, om_x_c;
+    } act;
 
     // pinned staging ring for the per-call metadata
     static constexpr int kSlots = 4;

@@ -124,14 +124,13 @@ cudaError_t launch_ffn_fused(const CUtensorMap &tmW1, const CUtensorMap &tmW2, c
                              const float *bo, int64_t M, int d_ff, float eps, int *err, cudaStream_t stream, int64_t *launches);
 
 // Flash-style attention on tcgen05 (d_head = 64) over the work items, then the merge of split items.  attn_kind: ATTN_SOFTMAX, or
-// ATTN_POINTWISE (weights SiLU(q.k / sqrt(d_h)) divided by the number of visible keys).  only_cand: skip tiles without a
-// candidate row (the last layer of a rank call, whose other rows nothing reads).
+// ATTN_POINTWISE (weights SiLU(q.k / sqrt(d_h)) divided by the number of visible keys).
 // tmQ: [rows, d] box 128 x 64; tmK / tmV: the call's transient K / V rows, box 64 x 64; tmPool: the pool
 // slab viewed as [pages * L * 2 * 64, d], box 64 x 64 (pass tmK when the call has no pool).
 cudaError_t launch_attention_tc(const CUtensorMap &tmQ, const CUtensorMap &tmK, const CUtensorMap &tmV, const CUtensorMap &tmPool,
                                 const AttnItem *items, int n_items, const AttnMerge *merges, int n_merges, const SeqDesc *seqs,
                                 const int32_t *pt, int n_layers, int layer, int d_model, const __nv_bfloat16 *q,
-                                const __nv_bfloat16 *k_lin, const __nv_bfloat16 *v_lin, int attn_kind, int only_cand, __nv_bfloat16 *out,
+                                const __nv_bfloat16 *k_lin, const __nv_bfloat16 *v_lin, int attn_kind, __nv_bfloat16 *out,
                                 float *partial, int *err, cudaStream_t stream, int64_t *launches);
 
 }  // namespace relaygr
