@@ -33,7 +33,7 @@ WORKLOAD = "config2: 4 layers, d_model 256, 4 heads x 64, FFN 1024, bf16; 32 use
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the config-2 rank step, from the ncu captures summarised
 # under profiles/ (None = no capture of the kernel as it stands).
-DRAM_TRAFFIC_BYTES = {"attention": 121.2e6, "gemm": 19.7e6}      # gemm: mean of QKV (9.9 MB) and the fused out-proj + feed-forward kernel (29.6 MB)
+DRAM_TRAFFIC_BYTES = {"attention": 123.4e6, "gemm": 19.7e6}      # gemm: mean of QKV (9.9 MB) and the fused out-proj + feed-forward kernel (29.6 MB)
 
 MIN_RANK_CALLS, MIN_FULL_CALLS = 500, 100       # individually timed calls behind every p50 / p99 of the main workload
 
@@ -237,6 +237,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--lat-calls", type=int, default=0, help="individually timed rank / full-recompute calls behind the percentiles "
+                    "(0 = at least 500 / 100; a small number keeps a run under a profiler short)")
     ap.add_argument("--no-legs", action="store_true", help="only the metric's own workload (no long-prefix, reload-tier and single-request legs)")
     ap.add_argument("--tier-population", type=int, default=4096, help="users of the reload-tier leg (their K/V sits in pinned DRAM; 16 MiB each)")
     ap.add_argument("--workload", type=int, default=2, choices=[2, 3, 4],
@@ -320,7 +322,7 @@ def main():
         return replicas.max_over_ranks(ms, dist, model.device)
 
     # ---- pre-infer (timed beside the metric) --------------------------------------------------------
-    pre_steps = max(20, min(40, args.steps // 10)) if sum(p_lens) < 200_000 else max(3, min(20, args.steps // 20))
+    pre_steps = max(3, min(20, args.steps // 20))        # 20 timed calls at the default --steps
     sampler = ClockSampler(local).start()
     pre_ms = preinfer_ms(torch, stream, workloads, built, pre_steps)
     pre_clocks = sampler.stop()
@@ -366,11 +368,11 @@ def main():
     value = world * n_cand / (ms_per_step * 1e-3)
 
     # one call at a time (stream idle before each call): per-call latency as a request sees it, and the host's share of it
-    n_lat = max(MIN_RANK_CALLS, min(args.steps, 2000)) if ms_per_step < 20 else max(100, min(args.steps, 500))
+    n_lat = args.lat_calls or (max(MIN_RANK_CALLS, min(args.steps, 2000)) if ms_per_step < 20 else max(100, min(args.steps, 500)))
     lat1, host_us = timed_calls(torch, stream, lambda i: pool.rank(built.dev_batches[i % nrot], scores), n_lat)
 
     # ---- full recompute of the same batches ---------------------------------------------------------
-    n_full = MIN_FULL_CALLS if ms_per_step < 20 else 20
+    n_full = args.lat_calls or (MIN_FULL_CALLS if ms_per_step < 20 else 20)
     full_lat, _ = timed_calls(torch, stream, lambda i: model.rank_full(built.dev_batches[i % nrot], scores), n_full, warmup=3)
 
     # ---- per-kernel timing of the rank step (events around every launch; separate from the timed region)
