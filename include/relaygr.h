@@ -167,6 +167,29 @@ int32_t relaygr_set_workspace(relaygr_ctx *ctx, void *dev, size_t bytes);
 #define RELAYGR_DEVSTATUS_BAD_INDEX    2
 int32_t relaygr_device_status(relaygr_ctx *ctx, void *stream, int32_t *out);
 
+/*
+ * Introspection, host only (no GPU, no ctx): the tensor-core attention work list that a
+ * bf16 call over users with the given lengths would launch on a GPU with `n_sms` SMs.
+ * mode 0 = pre-infer (queries: the prefix, causal), 1 = rank on cache (queries: short-term
+ * and candidate tokens; keys: the cached prefix, then the short-term tokens), 2 = full
+ * inference (queries: all tokens).  Lengths are host arrays [n_users]; short_len / cand_len
+ * are ignored for mode 0.  An item is one 128-row query tile of one head of one user
+ * against key blocks [blk0, blk1) of 64 keys; items run in list order, two per SM at a
+ * time.  A tile whose key range is split writes partial results that a merge combines.
+ *   items  [cap_items][8]  int32: user, head, q0, n_q, blk0, blk1, partial_slot (-1: none),
+ *                                  with_self (1: this item folds the candidates' own keys in)
+ *   merges [cap_merges][6] int32: user, head, q0, n_q, slot0, n_splits
+ * *n_items / *n_merges receive the counts; RELAYGR_E_NOSPACE if a capacity is too small
+ * (counts still set), RELAYGR_E_INVALID on bad arguments.  Used by the tests of the
+ * split policy (Section 3.2's ranking stage is latency-critical: a launch should not end in
+ * a wave of a few long items).
+ */
+int32_t relaygr_attention_plan(int32_t mode, int32_t n_users, const int32_t *prefix_len,
+                               const int32_t *short_len, const int32_t *cand_len,
+                               int32_t n_heads, int32_t n_sms,
+                               int32_t *items, int32_t cap_items, int32_t *n_items,
+                               int32_t *merges, int32_t cap_merges, int32_t *n_merges);
+
 /* ---- paged prefix-KV pool (Section 3.3 sliding window, Section 3.4 DRAM tier) ---------------- */
 
 /*

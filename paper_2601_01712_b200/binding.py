@@ -70,6 +70,7 @@ SIGNATURES = {
     "relaygr_workspace_bytes": (_I32, [_P, _I64, _I64, _I64, C.POINTER(_SZ)]),
     "relaygr_set_workspace": (_I32, [_P, _P, _SZ]),
     "relaygr_device_status": (_I32, [_P, _P, C.POINTER(_I32)]),
+    "relaygr_attention_plan": (_I32, [_I32, _I32, _P, _P, _P, _I32, _I32, _P, _I32, C.POINTER(_I32), _P, _I32, C.POINTER(_I32)]),
     "relaygr_kv_page_bytes": (_I32, [_P, C.POINTER(_SZ)]),
     "relaygr_kv_pool_create": (_I32, [_P, _P, _SZ, _P, _SZ, C.POINTER(_P)]),
     "relaygr_kv_pool_destroy": (_I32, [_P]),
@@ -173,6 +174,26 @@ def relaygr_device_status(ctx, stream=None) -> int:
     out = _I32()
     _check(lib().relaygr_device_status(ctx, stream, C.byref(out)))
     return out.value
+
+
+def relaygr_attention_plan(mode, prefix_len, short_len, cand_len, n_heads, n_sms):
+    """The attention work list of a call (host only).  Returns (items [n, 8], merges [m, 6]) as int32 numpy arrays."""
+    import numpy as np
+    n = len(prefix_len)
+    arr = lambda v: np.ascontiguousarray(np.asarray(v if v is not None else [0] * n, dtype=np.int32))
+    p, s_, c_ = arr(prefix_len), arr(short_len), arr(cand_len)
+    n_items, n_merges = _I32(), _I32()
+    cap_i, cap_m = 4096, 1024
+    while True:
+        items = np.zeros((cap_i, 8), dtype=np.int32)
+        merges = np.zeros((cap_m, 6), dtype=np.int32)
+        rc = lib().relaygr_attention_plan(mode, n, p.ctypes.data, s_.ctypes.data, c_.ctypes.data, n_heads, n_sms, items.ctypes.data, cap_i,
+                                          C.byref(n_items), merges.ctypes.data, cap_m, C.byref(n_merges))
+        if rc == E_NOSPACE:
+            cap_i, cap_m = max(cap_i, n_items.value), max(cap_m, n_merges.value)
+            continue
+        _check(rc)
+        return items[:n_items.value].copy(), merges[:n_merges.value].copy()
 
 
 def relaygr_kv_page_bytes(ctx) -> int:

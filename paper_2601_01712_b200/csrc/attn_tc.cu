@@ -2,9 +2,9 @@
 // pre-infer (causal over the user's own pages), rank on cache (prefix pages through the page
 // table + short-term rows + the candidate's own row) and full inference (linear K/V rows).
 //
-// One CTA = one work item: a 128-row query tile of one head of one user against a range of
-// that user's 64-key blocks (one block = one 64-token page of the pool, or 64 rows of the
-// call's transient K/V buffers; one 8 KB TMA box each for K and V).  Per block:
+// A work item = a 128-row query tile of one head of one user against a range of that user's
+// 64-key blocks (one block = one 64-token page of the pool, or 64 rows of the call's transient
+// K/V buffers; one 8 KB TMA box each for K and V).  Per block:
 //     S = Q K^T   tcgen05.mma M=128 N=64 K=64, operands in shared memory, S in TMEM
 //     softmax     128 threads, one row each: S row -> registers, running max, p = 2^(s c - m c),
 //                 bf16 P written back to TMEM
@@ -16,10 +16,20 @@
 // that some exponent may have exceeded 2^8 is the block maximum computed, the running maximum
 // raised, O rescaled in TMEM (after the pending PV has drained) and the block redone - so no
 // maximum is on the fast path, every exponent that is kept stays below 2^8, and rescales are rare.
+// A candidate's own key (it sees the prefix, the short-term tokens and itself) is one more block
+// of the same pipeline: the 64-row group of the call's K / V that holds the candidate's row, with
+// a diagonal mask (own_key_blocks).
 //
-// Warp roles (192 threads): warp 0 = TMA producer, warp 1 = TMEM owner + MMA issuer,
-// warps 2-5 = softmax / correction / epilogue (TMEM lane quadrant = warp index % 4).
-// Two CTAs per SM.
+// The kernel is persistent: two CTAs per SM, each drawing items from a counter until the list is
+// exhausted.  The TMA producer and the MMA issuer run on into the next item (its Q, its first K / V
+// tiles, its first two S) while the softmax warps finish the current one, so launch, set-up and
+// load latencies are paid once per CTA instead of once per item; barrier phases and pipeline
+// stages are counted over the CTA's running block index.
+//
+// Warp roles (192 threads): warp 0 = TMA producer (and the item counter), warp 1 = TMEM owner +
+// MMA issuer, warps 2-5 = softmax / correction / epilogue (TMEM lane quadrant = warp index % 4).
+#include <algorithm>
+
 #include "kernels.cuh"
 #include "tc_common.cuh"
 
@@ -42,9 +52,11 @@ constexpr int kPartStride = kDh + 4;                // floats per row of a split
 constexpr float kRowSumLimit = 256.f;               // a block's row sum above this: some p may exceed 2^8 -> redo against a raised maximum
 
 struct Bars {
-    uint64_t q_full;
+    uint64_t q_full, q_empty;
     uint64_t k_full[kStagesKV], k_empty[kStagesKV], v_full[kStagesKV], v_empty[kStagesKV];
     uint64_t s_full[2], p_full[2], p_free[2];
+    uint64_t item_full[2], item_empty[2];
+    int ring[2];                 // item indices on their way from the producer to the other warps (-1: no more)
     uint32_t tmem_slot;
     int abort_flag;
 };
@@ -100,11 +112,35 @@ __device__ __forceinline__ void exp2_fma_pipe(uint64_t x2, float &p0, float &p1)
     p1 = __uint_as_float(__float_as_uint(q1) + (__float_as_uint(r1) << 23));
 }
 
+// x if a == b, else y - as a select, never a branch (a per-lane `b` compared against every unrolled `a` otherwise
+// compiles to a jump table that diverges 32 ways)
+__device__ __forceinline__ uint32_t select_eq(int a, int b, uint32_t x, uint32_t y)
+{
+    uint32_t r;
+    asm("{\n .reg .pred p;\n setp.eq.s32 p, %1, %2;\n selp.b32 %0, %3, %4, p;\n}\n" : "=r"(r) : "r"(a), "r"(b), "r"(x), "r"(y));
+    return r;
+}
+
 __device__ __forceinline__ float max3(float a, float b, float c)
 {
     float d;
     asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
     return d;
+}
+
+// The candidates' own keys.  A candidate sees the prefix, the short-term tokens and itself: its own K / V row is not among
+// the key blocks above, so every 64-row group of the tile that holds a candidate row is appended to the item as one more
+// key block - rows self_row0 + q0 + 64 t .. + 63 of the call's K / V - with a diagonal mask: row r sees key r alone.
+// d0 = the first such group, n_diag = how many (0 when the item has no candidates, or is not the split that owns them).
+__device__ __forceinline__ void own_key_blocks(const AttnItem &it, const SeqDesc &sd, int &d0, int &n_diag)
+{
+    const int first_cand = max(0, sd.causal_end - (sd.q_pos0 + it.q0));      // first candidate row of the tile
+    d0 = 0;
+    n_diag = 0;
+    if (it.with_self && first_cand < it.n_q) {
+        d0 = first_cand / kKeys;
+        n_diag = (it.n_q + kKeys - 1) / kKeys - d0;
+    }
 }
 
 // kPointwise: pointwise aggregated attention (HSTU style) - the weight of a visible key is SiLU(q.k / sqrt(d_h)) and the
@@ -113,9 +149,9 @@ template <bool kPointwise>
 __global__ void __launch_bounds__(192, 2)
 attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmKlin,
                     const __grid_constant__ CUtensorMap tmVlin, const __grid_constant__ CUtensorMap tmPool,
-                    const AttnItem *__restrict__ items, const SeqDesc *__restrict__ seqs, const int32_t *__restrict__ pt,
-                    int n_layers, int layer, int d_model, const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restrict__ k_lin,
-                    const __nv_bfloat16 *__restrict__ v_lin, __nv_bfloat16 *__restrict__ out, float *__restrict__ partial, int *err)
+                    const AttnItem *__restrict__ items, int n_items, int *__restrict__ next_item, const SeqDesc *__restrict__ seqs,
+                    const int32_t *__restrict__ pt, int n_layers, int layer, int d_model, __nv_bfloat16 *__restrict__ out,
+                    float *__restrict__ partial, int *err)
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -127,7 +163,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     // set-up that touches nothing earlier kernels wrote; it may run while the previous kernel is still finishing
     if (threadIdx.x == 0) {
-        tc::mbar_init(&bars->q_full, 1);
+        tc::mbar_init(&bars->q_full, 1); tc::mbar_init(&bars->q_empty, 1);
         for (int s = 0; s < kStagesKV; ++s) {
             tc::mbar_init(&bars->k_full[s], 1); tc::mbar_init(&bars->k_empty[s], 1);
             tc::mbar_init(&bars->v_full[s], 1); tc::mbar_init(&bars->v_empty[s], 1);
@@ -135,6 +171,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         for (int b = 0; b < 2; ++b) {
             tc::mbar_init(&bars->s_full[b], 1);
             tc::mbar_init(&bars->p_full[b], 128); tc::mbar_init(&bars->p_free[b], 1);
+            tc::mbar_init(&bars->item_full[b], 1); tc::mbar_init(&bars->item_empty[b], 5);     // MMA warp + four softmax warps
         }
         tc::fence_mbar_init();
         tc::tma_prefetch_desc(&tmQ); tc::tma_prefetch_desc(&tmKlin); tc::tma_prefetch_desc(&tmVlin); tc::tma_prefetch_desc(&tmPool);
@@ -151,50 +188,90 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     tc::tc_fence_after();
     const uint32_t tmem_base = bars->tmem_slot;
     const bool live = bars->abort_flag == 0;                      // an earlier kernel gave up: do not pile on
-    const AttnItem it = items[blockIdx.x];
-    const SeqDesc sd = seqs[it.seq];
-    const int nb = it.blk1 - it.blk0;
-    const int n_paged_blocks = (sd.n_paged + kKeys - 1) / kKeys;      // = the user's page count
+
+    // Every role walks the same sequence of items: the producer draws an index from the launch's counter and passes it on
+    // through a two-slot ring.  `n` counts this CTA's items, `g` its key blocks since the kernel began: the stage of a K / V
+    // tile, the S / P buffer of a block and the phase of every barrier follow from g, so the pipelines run on across items.
+    // take_item(n): the index of this CTA's n-th item, or -1 when the list is exhausted (consumer side of the ring).
+    auto take_item = [&](int n, bool &ok) {
+        const int slot = n & 1;
+        ok = __all_sync(0xffffffffu, tc::mbar_wait(&bars->item_full[slot], (n >> 1) & 1, err));
+        const int idx = ok ? bars->ring[slot] : -1;
+        __syncwarp();
+        if (lane == 0) tc::mbar_arrive(&bars->item_empty[slot]);
+        return idx;
+    };
 
     if (!live) {
     } else if (warp == 0) {
         // ---------------------------------------------------------------- TMA producer
         if (lane == 0) {
-            tc::mbar_expect_tx(&bars->q_full, kQBytes);
-            tc::tma_load_2d(sQ, &tmQ, it.head * kDh, sd.q_row0 + it.q0, &bars->q_full);
-            for (int j = 0; j < nb; ++j) {
-                const int b = it.blk0 + j;
-                const int s = j % kStagesKV;
-                const uint32_t par = ((j / kStagesKV) & 1) ^ 1;
-                int ky, vy;
-                const CUtensorMap *mk, *mv;
-                if (b < n_paged_blocks) {
-                    const int page = pt[sd.pt_base + b];
-                    ky = ((page * n_layers + layer) * 2) * 64; vy = ky + 64;
-                    mk = &tmPool; mv = &tmPool;
-                } else {
-                    ky = vy = sd.lin_row0 + (b - n_paged_blocks) * kKeys;
-                    mk = &tmKlin; mv = &tmVlin;
+            int g = 0;
+            for (int n = 0;; ++n) {
+                const int slot = n & 1;
+                if (!tc::mbar_wait(&bars->item_empty[slot], ((n >> 1) & 1) ^ 1, err)) break;
+                int idx = atomicAdd(next_item, 1);
+                if (idx >= n_items) idx = -1;
+                bars->ring[slot] = idx;
+                tc::mbar_arrive(&bars->item_full[slot]);
+                if (idx < 0) break;
+                const AttnItem it = items[idx];
+                const SeqDesc sd = seqs[it.seq];
+                const int nb = it.blk1 - it.blk0;
+                int d0, n_diag;
+                own_key_blocks(it, sd, d0, n_diag);
+                const int n_paged_blocks = (sd.n_paged + kKeys - 1) / kKeys;      // = the user's page count
+                if (!tc::mbar_wait(&bars->q_empty, (n & 1) ^ 1, err)) break;       // the previous item's last Q K^T has read Q
+                tc::mbar_expect_tx(&bars->q_full, kQBytes);
+                tc::tma_load_2d(sQ, &tmQ, it.head * kDh, sd.q_row0 + it.q0, &bars->q_full);
+                bool ok = true;
+                for (int j = 0; j < nb + n_diag; ++j, ++g) {
+                    const int b = it.blk0 + j;
+                    const int s = g % kStagesKV;
+                    const uint32_t par = ((g / kStagesKV) & 1) ^ 1;
+                    int ky, vy;
+                    const CUtensorMap *mk, *mv;
+                    if (j >= nb) {                                       // the candidates' own rows
+                        ky = vy = sd.self_row0 + it.q0 + (d0 + j - nb) * kKeys;
+                        mk = &tmKlin; mv = &tmVlin;
+                    } else if (b < n_paged_blocks) {
+                        const int page = pt[sd.pt_base + b];
+                        ky = ((page * n_layers + layer) * 2) * 64; vy = ky + 64;
+                        mk = &tmPool; mv = &tmPool;
+                    } else {
+                        ky = vy = sd.lin_row0 + (b - n_paged_blocks) * kKeys;
+                        mk = &tmKlin; mv = &tmVlin;
+                    }
+                    if (!(ok = tc::mbar_wait(&bars->k_empty[s], par, err))) break;
+                    tc::mbar_expect_tx(&bars->k_full[s], kKVBytes);
+                    tc::tma_load_2d(sK + s * kKVBytes, mk, it.head * kDh, ky, &bars->k_full[s]);
+                    if (!(ok = tc::mbar_wait(&bars->v_empty[s], par, err))) break;
+                    tc::mbar_expect_tx(&bars->v_full[s], kKVBytes);
+                    tc::tma_load_2d(sV + s * kKVBytes, mv, it.head * kDh, vy, &bars->v_full[s]);
                 }
-                if (!tc::mbar_wait(&bars->k_empty[s], par, err)) break;
-                tc::mbar_expect_tx(&bars->k_full[s], kKVBytes);
-                tc::tma_load_2d(sK + s * kKVBytes, mk, it.head * kDh, ky, &bars->k_full[s]);
-                if (!tc::mbar_wait(&bars->v_empty[s], par, err)) break;
-                tc::mbar_expect_tx(&bars->v_full[s], kKVBytes);
-                tc::tma_load_2d(sV + s * kKVBytes, mv, it.head * kDh, vy, &bars->v_full[s]);
+                if (!ok) break;
             }
         }
     } else if (warp == 1) {
         // ---------------------------------------------------------------- MMA issuer (the whole warp walks the loop so
         // that addresses and descriptors stay warp-uniform; one elected lane issues the tcgen05 instructions)
-        {
-            constexpr uint32_t idesc_qk = tc::make_idesc(128, kKeys, 0, 0);   // Q, K both K-major
-            constexpr uint32_t idesc_pv = tc::make_idesc(128, kDh, 0, 1);     // P from TMEM, V MN-major
-            const uint64_t qdesc = tc::smem_desc_sw128(tc::smem_u32(sQ));
-            bool ok = tc::mbar_wait(&bars->q_full, 0, err);
-            auto issue_qk = [&](int j) {        // S[j & 1] = Q K(j)^T
-                const int s = j % kStagesKV, b = j & 1;
-                if (!tc::mbar_wait(&bars->k_full[s], (j / kStagesKV) & 1, err)) return false;
+        constexpr uint32_t idesc_qk = tc::make_idesc(128, kKeys, 0, 0);   // Q, K both K-major
+        constexpr uint32_t idesc_pv = tc::make_idesc(128, kDh, 0, 1);     // P from TMEM, V MN-major
+        const uint64_t qdesc = tc::smem_desc_sw128(tc::smem_u32(sQ));
+        int g = 0;
+        bool ok = true;
+        for (int n = 0; ok; ++n) {
+            const int idx = take_item(n, ok);
+            if (idx < 0) break;
+            const AttnItem it = items[idx];
+            int d0, n_diag;
+            own_key_blocks(it, seqs[it.seq], d0, n_diag);
+            const int nb = it.blk1 - it.blk0 + n_diag;         // key blocks of the item, the candidates' own included
+            ok = tc::mbar_wait(&bars->q_full, n & 1, err);
+            if (!ok) break;
+            auto issue_qk = [&](int j) {        // S[(g + j) & 1] = Q K(j)^T; the item's last one also hands Q back
+                const int gb = g + j, s = gb % kStagesKV, b = gb & 1;
+                if (!tc::mbar_wait(&bars->k_full[s], (gb / kStagesKV) & 1, err)) return false;
                 tc::tc_fence_after();
                 const uint64_t kdesc = tc::smem_desc_sw128(tc::smem_u32(sK + s * kKVBytes));
                 if (tc::elect_one()) {
@@ -203,58 +280,79 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                         tc::mma_ss(tmem_base + kColS + b * kKeys, qdesc + 2 * k, kdesc + 2 * k, idesc_qk, k != 0);
                     tc::mma_commit(&bars->s_full[b]);
                     tc::mma_commit(&bars->k_empty[s]);
+                    if (j == nb - 1) tc::mma_commit(&bars->q_empty);
                 }
                 __syncwarp();
                 return true;
             };
-            if (ok && nb > 0) ok = issue_qk(0);
+            // Both S buffers are free here: every P V of the previous item has been issued, each of them after the softmax
+            // threads had taken the S of its block into registers.
+            if (nb == 0) {
+                if (lane == 0) tc::mbar_arrive(&bars->q_empty);
+                __syncwarp();
+            }
+            if (nb > 0) ok = issue_qk(0);
             if (ok && nb > 1) ok = issue_qk(1);
             for (int j = 0; j < nb && ok; ++j) {
-                const int s = j % kStagesKV, b = j & 1;
-                if (!tc::mbar_wait(&bars->p_full[b], (j >> 1) & 1, err)) break;
-                if (!tc::mbar_wait(&bars->v_full[s], (j / kStagesKV) & 1, err)) break;
+                const int gb = g + j, s = gb % kStagesKV, b = gb & 1;
+                if (!(ok = tc::mbar_wait(&bars->p_full[b], (gb >> 1) & 1, err))) break;
+                if (!(ok = tc::mbar_wait(&bars->v_full[s], (gb / kStagesKV) & 1, err))) break;
                 tc::tc_fence_after();
                 const uint64_t vdesc = tc::smem_desc_sw128(tc::smem_u32(sV + s * kKVBytes));
                 if (tc::elect_one()) {
 #pragma unroll
                     for (int k = 0; k < kKeys / 16; ++k)      // 16 keys per instruction: 8 TMEM columns of P, 2048 bytes of V
                         tc::mma_ts(tmem_base + kColO, tmem_base + kColP + b * (kKeys / 2) + 8 * k, vdesc + 128 * k, idesc_pv, (j | k) != 0);
-                    tc::mma_commit(&bars->p_free[b]);          // P[b] consumed; also "O holds blocks 0..j"
+                    tc::mma_commit(&bars->p_free[b]);          // P[b] consumed; also "O holds blocks 0..j of the item"
                     tc::mma_commit(&bars->v_empty[s]);
                 }
                 __syncwarp();
                 // QK(j + 2) follows PV(j) in issue order, and a commit covers everything issued before it: a softmax
                 // thread that sees s_full of block j + 2 also knows that P[b] has been consumed.  S[b] is free as well:
-                // P(j) was published only after the softmax had taken S(j) into registers.
+                // P(j) was published only after the softmax had taken S(j) into registers.  (The first P V of the next
+                // item overwrites O: it waits for that item's first P, which every softmax thread publishes only after
+                // its epilogue has read O.)
                 if (j + 2 < nb) ok = issue_qk(j + 2);
             }
+            g += nb;
         }
     } else {
         // ---------------------------------------------------------------- softmax / correction / epilogue
         const int quad = warp & 3;
-        const int r = quad * 32 + lane;                      // row of the tile this thread owns
         const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
+        const float c = 0.125f * 1.4426950408889634f;        // 1/sqrt(64) * log2(e)
+        int g = 0;
+        bool ok = true;
+        for (int n = 0; ok; ++n) {
+        const int idx = take_item(n, ok);
+        if (idx < 0) break;
+        const AttnItem it = items[idx];
+        const SeqDesc sd = seqs[it.seq];
+        int d0, n_diag;
+        own_key_blocks(it, sd, d0, n_diag);
+        const int nb_keys = it.blk1 - it.blk0, nb = nb_keys + n_diag;     // the candidates' own keys come last
+        const int n_paged_blocks = (sd.n_paged + kKeys - 1) / kKeys;      // = the user's page count
+        const int r = quad * 32 + lane;                      // row of the tile this thread owns
         const int tpos = sd.q_pos0 + it.q0 + r;              // sequence position of the row
         const bool is_cand = tpos >= sd.causal_end;
         const int lim = is_cand ? sd.causal_end - 1 : tpos;  // last visible key position
         const int tile_min_lim = (sd.q_pos0 + it.q0 >= sd.causal_end) ? sd.causal_end - 1 : sd.q_pos0 + it.q0;
-        const float c = 0.125f * 1.4426950408889634f;        // 1/sqrt(64) * log2(e)
         float m = -INFINITY, l = 0.f;
-        bool ok = true;
         // a warp whose 32 rows all lie past the tile's last row keeps the hand-shakes going but takes no exponentials:
         // its rows of P (and of O) hold whatever TMEM held, which only ever reaches those same, unused, rows
         const bool warp_live = quad * 32 < it.n_q;
 
         for (int j = 0; j < nb && ok; ++j) {
-            const int blk = it.blk0 + j, b = j & 1;
+            const int blk = it.blk0 + j, gb = g + j, b = gb & 1;
             const bool paged = blk < n_paged_blocks;
             const int kidx0 = paged ? blk * kKeys : (blk - n_paged_blocks) * kKeys;    // index of the block's first key in its source
             const int kpos0 = paged ? kidx0 : sd.lin_pos0 + kidx0;                     // its sequence position
             const int n_valid = min(kKeys, (paged ? sd.n_paged : sd.n_lin) - kidx0);
-            const bool need_mask = (n_valid < kKeys) || (kpos0 + kKeys - 1 > tile_min_lim);
+            const bool own_keys = j >= nb_keys;              // a block of the candidates' own keys (values above unused)
+            const bool need_mask = !own_keys && ((n_valid < kKeys) || (kpos0 + kKeys - 1 > tile_min_lim));
             const int jmax = min(n_valid, lim - kpos0 + 1);  // keys jj < jmax of this block are visible to this row
 
-            ok = __all_sync(0xffffffffu, tc::mbar_wait(&bars->s_full[b], (j >> 1) & 1, err));
+            ok = __all_sync(0xffffffffu, tc::mbar_wait(&bars->s_full[b], (gb >> 1) & 1, err));
             if (!ok) break;
             tc::tc_fence_after();
             if (!warp_live) {
@@ -273,6 +371,16 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 for (int i = 0; i < 32; ++i) {
                     if (i >= jmax) s0[i] = kPointwise ? 0u : 0xff800000u;      // -inf (softmax) or a logit of 0: SiLU(0) = 0
                     if (32 + i >= jmax) s1[i] = kPointwise ? 0u : 0xff800000u;
+                }
+            }
+            if (own_keys) {
+                // a candidate row of this 64-row group sees its own key (the diagonal of the block) and nothing else;
+                // every other row of the tile sees nothing here
+                const int own = is_cand ? r - (d0 + j - nb_keys) * kKeys : -1;
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                    s0[i] = select_eq(i, own, s0[i], kPointwise ? 0u : 0xff800000u);
+                    s1[i] = select_eq(32 + i, own, s1[i], kPointwise ? 0u : 0xff800000u);
                 }
             }
             if constexpr (kPointwise) {
@@ -359,7 +467,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 }
                 if (j > 0 && __any_sync(0xffffffffu, raise)) {
                     // correction: O must hold blocks 0..j-1 completely before it is rescaled
-                    ok = __all_sync(0xffffffffu, tc::mbar_wait(&bars->p_free[(j - 1) & 1], ((j - 1) >> 1) & 1, err));
+                    ok = __all_sync(0xffffffffu, tc::mbar_wait(&bars->p_free[(gb - 1) & 1], ((gb - 1) >> 1) & 1, err));
                     if (!ok) break;
                     tc::tc_fence_after();
 #pragma unroll 1
@@ -380,8 +488,10 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             tc::mbar_arrive(&bars->p_full[b]);     // P(j) (and any correction of O) is in TMEM
         }
 
-        // ---- epilogue: O / l (plus the candidate's own key), or the split partial
-        if (ok && nb > 0) ok = __all_sync(0xffffffffu, tc::mbar_wait(&bars->p_free[(nb - 1) & 1], ((nb - 1) >> 1) & 1, err));
+        if (!ok) break;
+        // ---- epilogue: O / l, or the split partial
+        if (nb > 0) ok = __all_sync(0xffffffffu, tc::mbar_wait(&bars->p_free[(g + nb - 1) & 1], ((g + nb - 1) >> 1) & 1, err));
+        if (!ok) break;
         tc::tc_fence_after();
         if (ok && warp_live) {
             float o[kDh];
@@ -400,48 +510,6 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             }
             const bool row_ok = r < it.n_q;
             const int64_t row = (int64_t)sd.q_row0 + it.q0 + r;
-            if (row_ok && is_cand && it.with_self) {
-                // the candidate's own key / value row, folded into the running softmax on CUDA cores
-                const int64_t self = (int64_t)sd.self_row0 + it.q0 + r;
-                const uint4 *qp = reinterpret_cast<const uint4 *>(q + row * d_model + it.head * kDh);
-                const uint4 *kp = reinterpret_cast<const uint4 *>(k_lin + self * d_model + it.head * kDh);
-                const uint4 *vp = reinterpret_cast<const uint4 *>(v_lin + self * d_model + it.head * kDh);
-                float dot = 0.f;
-#pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    const uint4 a = qp[i], bq = kp[i];
-                    const __nv_bfloat162 *a2 = reinterpret_cast<const __nv_bfloat162 *>(&a);
-                    const __nv_bfloat162 *b2 = reinterpret_cast<const __nv_bfloat162 *>(&bq);
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const float2 fa = __bfloat1622float2(a2[e]), fb = __bfloat1622float2(b2[e]);
-                        dot = fmaf(fa.x, fb.x, dot); dot = fmaf(fa.y, fb.y, dot);
-                    }
-                }
-                float al, ps;
-                if constexpr (kPointwise) {
-                    const float z = dot * 0.125f;
-                    al = 1.f;
-                    ps = z / (1.f + __expf(-z));
-                } else {
-                    const float mn = fmaxf(m, dot);
-                    al = (m == -INFINITY) ? 0.f : ex2((m - mn) * c);
-                    ps = ex2((dot - mn) * c);
-                    l = l * al + ps;
-                    m = mn;
-                }
-#pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    const uint4 vv = vp[i];
-                    const __nv_bfloat162 *v2 = reinterpret_cast<const __nv_bfloat162 *>(&vv);
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const float2 fv = __bfloat1622float2(v2[e]);
-                        o[i * 8 + 2 * e] = fmaf(o[i * 8 + 2 * e], al, ps * fv.x);
-                        o[i * 8 + 2 * e + 1] = fmaf(o[i * 8 + 2 * e + 1], al, ps * fv.y);
-                    }
-                }
-            }
             if constexpr (kPointwise) {
                 // the normaliser is the number of keys the row may see (every key position below its limit, plus itself for
                 // a candidate); a split item hands it over as l with m = 0, so that the merge of partials needs no change
@@ -470,6 +538,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 }
             }
         }
+        g += nb;
+        }   // items
     }
     tc::tc_fence_before();
     __syncthreads();
@@ -512,9 +582,8 @@ attention_merge_kernel(const AttnMerge *__restrict__ merges, const SeqDesc *__re
 
 cudaError_t launch_attention_tc(const CUtensorMap &tmQ, const CUtensorMap &tmK, const CUtensorMap &tmV, const CUtensorMap &tmPool,
                                 const AttnItem *items, int n_items, const AttnMerge *merges, int n_merges, const SeqDesc *seqs,
-                                const int32_t *pt, int n_layers, int layer, int d_model, const __nv_bfloat16 *q,
-                                const __nv_bfloat16 *k_lin, const __nv_bfloat16 *v_lin, int attn_kind, __nv_bfloat16 *out,
-                                float *partial, int *err, cudaStream_t stream, int64_t *launches)
+                                const int32_t *pt, int n_layers, int layer, int d_model, int attn_kind, __nv_bfloat16 *out,
+                                float *partial, int *next_item, int n_sms, int *err, cudaStream_t stream, int64_t *launches)
 {
     if (n_items == 0) return cudaSuccess;
     static PerDeviceValue attr_set;
@@ -529,8 +598,9 @@ cudaError_t launch_attention_tc(const CUtensorMap &tmQ, const CUtensorMap &tmK, 
     }
     *launches += 1;
     auto kernel = attn_kind == ATTN_POINTWISE ? attention_tc_kernel<true> : attention_tc_kernel<false>;
-    cudaError_t e = launch_dependent(kernel, dim3(n_items), dim3(192), (size_t)kSmemBytes, stream, 1, tmQ, tmK, tmV, tmPool, items,
-                                     seqs, pt, n_layers, layer, d_model, q, k_lin, v_lin, out, partial, err);
+    const int grid = std::min(n_items, 2 * std::max(1, n_sms));       // two CTAs per SM, each drawing items until none is left
+    cudaError_t e = launch_dependent(kernel, dim3(grid), dim3(192), (size_t)kSmemBytes, stream, 1, tmQ, tmK, tmV, tmPool, items,
+                                     n_items, next_item, seqs, pt, n_layers, layer, d_model, out, partial, err);
     if (e != cudaSuccess || n_merges == 0) return e;
     *launches += 1;
     return launch_dependent(attention_merge_kernel, dim3(n_merges, kQTile / 8), dim3(256), 0, stream, 1, merges, seqs, partial, d_model, out);

@@ -135,7 +135,7 @@ WorkspaceLayout Forward::layout(int64_t rows, int64_t users, int64_t pages) cons
     l.partial = take(l.partial_bytes);
     const size_t n_items = (size_t)cfg.n_heads * ((size_t)rows / 128 + (size_t)users + 1) + 2 * (size_t)kMaxSplitTiles;
     // two descriptor arrays and two work lists: all rows, and the candidate rows of the last layer
-    l.meta_bytes = 4 * (((size_t)users + 1) * 5 + 2 * (size_t)users * (sizeof(SeqDesc) / 4) + (size_t)pages + 2 * n_items * (sizeof(AttnItem) / 4) + 64);
+    l.meta_bytes = 4 * (((size_t)users + 1) * 5 + 2 * (size_t)users * (sizeof(SeqDesc) / 4) + (size_t)pages + 2 * n_items * (sizeof(AttnItem) / 4) + (size_t)cfg.n_layers + 64);
     l.meta = take(l.meta_bytes);
     l.total = at;
     return l;
@@ -207,57 +207,8 @@ int Forward::run_t(const CallDesc &call, float *scores, cudaStream_t stream, std
     // projection, attention, output projection and feed-forward run on those rows alone.
     const bool compact_last = kTensor && !preinfer;
 
-    // ---- tensor-core attention work items: one per (user, head, 128-row tile[, KV split]) of the rows in `seqs`
     auto build_items = [&](const std::vector<SeqDesc> &seqs, std::vector<AttnItem> &items, std::vector<AttnMerge> &merges) {
-        struct Tile { int seq, q0, n_q, nb; };
-        std::vector<Tile> tiles;
-        for (int u = 0; u < (int)seqs.size(); ++u) {
-            const SeqDesc &sd = seqs[(size_t)u];
-            const int nPB = (sd.n_paged + 63) / 64, nLB = (sd.n_lin + 63) / 64;      // key blocks of 64 (one page each)
-            for (int q0 = 0; q0 < sd.n_q; q0 += 128) {
-                const int n_q = std::min(128, sd.n_q - q0);
-                const int tp1 = sd.q_pos0 + q0 + n_q - 1;
-                const int kmax = tp1 < sd.causal_end ? tp1 : sd.causal_end - 1;      // last key position any row of the tile sees
-                int nb = 0;
-                if (kmax >= 0) {
-                    const int pb = sd.n_paged > 0 ? std::min(nPB, kmax / 64 + 1) : 0;
-                    int lb = 0;
-                    if (pb == nPB && sd.n_lin > 0 && kmax >= sd.lin_pos0) lb = std::min(nLB, (kmax - sd.lin_pos0) / 64 + 1);
-                    nb = pb + lb;
-                }
-                tiles.push_back({u, q0, n_q, nb});
-            }
-        }
-        // split long key ranges when there are too few tiles to fill the GPU
-        const int64_t base = (int64_t)tiles.size() * H;
-        const int64_t target = 2 * (int64_t)n_sms;
-        int want = base > 0 && base < target ? (int)((target + base - 1) / base) : 1;
-        int part_slot = 0;
-        // costliest first (key blocks x softmax warps with live rows), so that the cheap partial tiles fill the last wave;
-        // ties keep a user's tiles together (they share K / V through L2)
-        std::sort(tiles.begin(), tiles.end(), [](const Tile &x, const Tile &y) {
-            const int64_t cx = (int64_t)x.nb * ((x.n_q + 31) / 32), cy = (int64_t)y.nb * ((y.n_q + 31) / 32);
-            if (cx != cy) return cx > cy;
-            if (x.seq != y.seq) return x.seq < y.seq;
-            return x.q0 < y.q0;
-        });
-        for (const Tile &t : tiles) {
-            int ns = std::max(1, std::min(want, t.nb / 8));          // at least 8 key blocks (512 keys) per split
-            if (ns > 1 && part_slot + ns * H > kMaxSplitTiles) ns = 1;
-            const bool has_cand = seqs[(size_t)t.seq].q_pos0 + t.q0 + t.n_q > seqs[(size_t)t.seq].causal_end;
-            for (int h = 0; h < H; ++h) {
-                if (ns == 1) {
-                    items.push_back({t.seq, h, t.q0, t.n_q, 0, t.nb, -1, has_cand ? 1 : 0});
-                } else {
-                    merges.push_back({t.seq, h, t.q0, t.n_q, part_slot, ns});
-                    for (int i = 0; i < ns; ++i) {
-                        const int b0 = (int)((int64_t)t.nb * i / ns), b1 = (int)((int64_t)t.nb * (i + 1) / ns);
-                        items.push_back({t.seq, h, t.q0, t.n_q, b0, b1, part_slot + i, (i == 0 && has_cand) ? 1 : 0});
-                    }
-                    part_slot += ns;
-                }
-            }
-        }
+        build_attention_worklist(seqs, H, n_sms, kMaxSplitTiles, items, merges);
     };
 
     // ---- metadata blob: row_off | seg_off x3 | score_off | SeqDesc[] | page table | attention items [| the same for the last layer]
@@ -296,6 +247,9 @@ int Forward::run_t(const CallDesc &call, float *scores, cudaStream_t stream, std
             if (!merges_c.empty()) o_merges_c = put(reinterpret_cast<const int32_t *>(merges_c.data()), merges_c.size() * (sizeof(AttnMerge) / 4));
         }
     }
+    // one item counter per layer's attention launch (the persistent kernel draws its work from it), zeroed by this upload
+    const std::vector<int32_t> zeros((size_t)L, 0);
+    const size_t o_ctr = kTensor ? put(zeros.data(), zeros.size()) : 0;
     if (blob.size() * 4 > lay.meta_bytes) { err = "internal: metadata larger than its workspace region"; return RELAYGR_E_NOSPACE; }
     int rc = upload(blob, lay.meta, stream, err);
     if (rc) return rc;
@@ -446,8 +400,8 @@ int Forward::run_t(const CallDesc &call, float *scores, cudaStream_t stream, std
             cudaEvent_t pe = prof_begin(stream);
             if constexpr (kTensor)
                 e = launch_attention_tc(tm_q, tm_k, tm_v, tm_pool, items_m, n_items_m, merges_m, n_merges_m, seqs_m, meta + o_pt, L,
-                                        l, d, q, kl, vl, cfg.attn_kind, att, reinterpret_cast<float *>(ws + lay.partial), d_status,
-                                        stream, &launches);
+                                        l, d, cfg.attn_kind, att, reinterpret_cast<float *>(ws + lay.partial),
+                                        reinterpret_cast<int *>(ws + lay.meta) + o_ctr + l, n_sms, d_status, stream, &launches);
             else
                 e = launch_attention_simt<T>(q, kl, vl, paged, d_seqs, d_row_off, B, R, H, cfg.d_head, cfg.attn_kind, att, stream, &launches);
             prof_end(KC_ATTENTION, pe, stream);

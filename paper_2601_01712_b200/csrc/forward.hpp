@@ -17,6 +17,10 @@ namespace relaygr {
 
 enum CallMode { MODE_PREINFER = 0, MODE_RANK = 1, MODE_FULL = 2 };
 
+// The attention work list of one call (host only): items in launch order, and the merges of split items.
+void build_attention_worklist(const std::vector<SeqDesc> &seqs, int n_heads, int n_sms, int64_t max_split_tiles,
+                              std::vector<AttnItem> &items, std::vector<AttnMerge> &merges);
+
 struct CallDesc {
     int mode = MODE_RANK;
     std::vector<SeqDesc> seqs;

@@ -127,10 +127,11 @@ cudaError_t launch_ffn_fused(const CUtensorMap &tmW1, const CUtensorMap &tmW2, c
 // ATTN_POINTWISE (weights SiLU(q.k / sqrt(d_h)) divided by the number of visible keys).
 // tmQ: [rows, d] box 128 x 64; tmK / tmV: the call's transient K / V rows, box 64 x 64; tmPool: the pool
 // slab viewed as [pages * L * 2 * 64, d], box 64 x 64 (pass tmK when the call has no pool).
+// The kernel is persistent: min(n_items, 2 x n_sms) CTAs draw item indices from *next_item, a device counter that must be
+// zero when the kernel starts and belongs to this launch alone (the kernel leaves it non-zero).
 cudaError_t launch_attention_tc(const CUtensorMap &tmQ, const CUtensorMap &tmK, const CUtensorMap &tmV, const CUtensorMap &tmPool,
                                 const AttnItem *items, int n_items, const AttnMerge *merges, int n_merges, const SeqDesc *seqs,
-                                const int32_t *pt, int n_layers, int layer, int d_model, const __nv_bfloat16 *q,
-                                const __nv_bfloat16 *k_lin, const __nv_bfloat16 *v_lin, int attn_kind, __nv_bfloat16 *out,
-                                float *partial, int *err, cudaStream_t stream, int64_t *launches);
+                                const int32_t *pt, int n_layers, int layer, int d_model, int attn_kind, __nv_bfloat16 *out,
+                                float *partial, int *next_item, int n_sms, int *err, cudaStream_t stream, int64_t *launches);
 
 }  // namespace relaygr

@@ -140,6 +140,42 @@ int32_t relaygr_device_status(relaygr_ctx *ctx, void *stream, int32_t *out)
     return ctx->fwd.device_status((cudaStream_t)stream, out, g_err);
 }
 
+int32_t relaygr_attention_plan(int32_t mode, int32_t n_users, const int32_t *prefix_len, const int32_t *short_len,
+                               const int32_t *cand_len, int32_t n_heads, int32_t n_sms, int32_t *items, int32_t cap_items,
+                               int32_t *n_items, int32_t *merges, int32_t cap_merges, int32_t *n_merges)
+{
+    if (mode < 0 || mode > 2 || n_users < 0 || n_heads < 1 || n_sms < 1 || !n_items || !n_merges || cap_items < 0 || cap_merges < 0 ||
+        (n_users > 0 && !prefix_len) || (mode != 0 && n_users > 0 && (!short_len || !cand_len)) || (cap_items > 0 && !items) ||
+        (cap_merges > 0 && !merges))
+        return fail(RELAYGR_E_INVALID, "bad argument");
+    // the same descriptors as relaygr_preinfer / relaygr_rank / relaygr_rank_full build (rows and page-table bases do not
+    // enter the plan; only lengths and positions do)
+    std::vector<SeqDesc> seqs;
+    int64_t row = 0;
+    for (int i = 0; i < n_users; ++i) {
+        const int P = prefix_len[i], S = mode == 0 ? 0 : short_len[i], C = mode == 0 ? 0 : cand_len[i];
+        if (P < 0 || S < 0 || C < 0 || row + (int64_t)P + S + C > INT32_MAX) return fail(RELAYGR_E_INVALID, "bad length");
+        SeqDesc s{};
+        s.q_row0 = (int32_t)row;
+        if (mode == 0) { s.n_q = P; s.q_pos0 = 0; s.n_paged = P; s.n_lin = 0; s.lin_pos0 = P; s.causal_end = P; }
+        else if (mode == 1) { s.n_q = S + C; s.q_pos0 = P; s.n_paged = P; s.n_lin = S; s.lin_pos0 = P; s.causal_end = P + S; }
+        else { s.n_q = P + S + C; s.q_pos0 = 0; s.n_paged = 0; s.n_lin = P + S; s.lin_pos0 = 0; s.causal_end = P + S; }
+        s.lin_row0 = s.self_row0 = s.q_row0;
+        row += s.n_q;
+        seqs.push_back(s);
+    }
+    std::vector<AttnItem> it;
+    std::vector<AttnMerge> mg;
+    build_attention_worklist(seqs, n_heads, n_sms, Forward::kMaxSplitTiles, it, mg);
+    *n_items = (int32_t)it.size();
+    *n_merges = (int32_t)mg.size();
+    if ((int64_t)it.size() > cap_items || (int64_t)mg.size() > cap_merges) return fail(RELAYGR_E_NOSPACE, "plan larger than the arrays given");
+    static_assert(sizeof(AttnItem) == 8 * sizeof(int32_t) && sizeof(AttnMerge) == 6 * sizeof(int32_t), "layout of the plan arrays");
+    if (!it.empty()) std::memcpy(items, it.data(), it.size() * sizeof(AttnItem));
+    if (!mg.empty()) std::memcpy(merges, mg.data(), mg.size() * sizeof(AttnMerge));
+    return RELAYGR_OK;
+}
+
 int32_t relaygr_profile_enable(relaygr_ctx *ctx, int32_t on)
 {
     if (!ctx) return fail(RELAYGR_E_INVALID, "ctx is NULL");
