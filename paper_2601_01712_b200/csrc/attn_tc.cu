@@ -337,20 +337,31 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         const bool is_cand = tpos >= sd.causal_end;
         const int lim = is_cand ? sd.causal_end - 1 : tpos;  // last visible key position
         const int tile_min_lim = (sd.q_pos0 + it.q0 >= sd.causal_end) ? sd.causal_end - 1 : sd.q_pos0 + it.q0;
+        // Blocks [0, n_clean) of the user are complete (64 keys) and visible to every row of the tile: no mask, and none of
+        // the per-block position arithmetic, which otherwise sits as a dependent chain between publishing P(j) and polling
+        // for S(j + 1).  Pages come first in the block order, then the 64-row groups of linear keys.
+        int n_clean = min(sd.n_paged / kKeys, (tile_min_lim + 1) / kKeys);
+        if (n_clean == n_paged_blocks && tile_min_lim >= sd.lin_pos0) n_clean += min(sd.n_lin, tile_min_lim + 1 - sd.lin_pos0) / kKeys;
+        n_clean -= it.blk0;                                   // relative to the item's first block
         float m = -INFINITY, l = 0.f;
         // a warp whose 32 rows all lie past the tile's last row keeps the hand-shakes going but takes no exponentials:
         // its rows of P (and of O) hold whatever TMEM held, which only ever reaches those same, unused, rows
         const bool warp_live = quad * 32 < it.n_q;
 
         for (int j = 0; j < nb && ok; ++j) {
-            const int blk = it.blk0 + j, gb = g + j, b = gb & 1;
-            const bool paged = blk < n_paged_blocks;
-            const int kidx0 = paged ? blk * kKeys : (blk - n_paged_blocks) * kKeys;    // index of the block's first key in its source
-            const int kpos0 = paged ? kidx0 : sd.lin_pos0 + kidx0;                     // its sequence position
-            const int n_valid = min(kKeys, (paged ? sd.n_paged : sd.n_lin) - kidx0);
-            const bool own_keys = j >= nb_keys;              // a block of the candidates' own keys (values above unused)
-            const bool need_mask = !own_keys && ((n_valid < kKeys) || (kpos0 + kKeys - 1 > tile_min_lim));
-            const int jmax = min(n_valid, lim - kpos0 + 1);  // keys jj < jmax of this block are visible to this row
+            const int gb = g + j, b = gb & 1;
+            const bool own_keys = j >= nb_keys;              // a block of the candidates' own keys
+            bool need_mask = false;
+            int jmax = kKeys;                                // keys jj < jmax of this block are visible to this row
+            if (j >= n_clean && !own_keys) {
+                const int blk = it.blk0 + j;
+                const bool paged = blk < n_paged_blocks;
+                const int kidx0 = paged ? blk * kKeys : (blk - n_paged_blocks) * kKeys;    // index of the block's first key in its source
+                const int kpos0 = paged ? kidx0 : sd.lin_pos0 + kidx0;                     // its sequence position
+                const int n_valid = min(kKeys, (paged ? sd.n_paged : sd.n_lin) - kidx0);
+                need_mask = (n_valid < kKeys) || (kpos0 + kKeys - 1 > tile_min_lim);
+                jmax = min(n_valid, lim - kpos0 + 1);
+            }
 
             ok = __all_sync(0xffffffffu, tc::mbar_wait(&bars->s_full[b], (gb >> 1) & 1, err));
             if (!ok) break;
