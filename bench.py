@@ -33,7 +33,7 @@ WORKLOAD = "config2: 4 layers, d_model 256, 4 heads x 64, FFN 1024, bf16; 32 use
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the config-2 rank step, from the ncu captures summarised
 # under profiles/ (None = no capture of the kernel as it stands).
-DRAM_TRAFFIC_BYTES = {"attention": 123.4e6, "gemm": 19.7e6}      # gemm: mean of QKV (9.9 MB) and the fused out-proj + feed-forward kernel (29.6 MB)
+DRAM_TRAFFIC_BYTES = {"attention": 117.3e6, "gemm": 19.7e6}      # gemm: mean of QKV (9.9 MB) and the fused out-proj + feed-forward kernel (29.6 MB)
 
 MIN_RANK_CALLS, MIN_FULL_CALLS = 500, 100       # individually timed calls behind every p50 / p99 of the main workload
 
